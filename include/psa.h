@@ -1,0 +1,123 @@
+/*
+ * psa.h -- C ABI of the B200 (sm_100a) parameterized-stripe-attention library.
+ *
+ * The library computes the forward pass of block-sparse video attention whose
+ * per-head mask is generated from six integers M(T_w, T_o, T_s, S_w, S_o, S_s)
+ * (Section 3.2, "Unified Representation", and Algorithm 1), applied at PSABlock
+ * granularity (Section 3.2, "Hardware-Aware Design") on the 3D-padded block grid
+ * (Section 3.2, "3D-Padding"), followed by flash-style attention over the
+ * surviving blocks (Appendix B, Algorithm 2).
+ *
+ * Conventions shared by every call
+ *   - Tokens are in frame-major, row-major order i = t*H*W + h*W + w (Appendix D,
+ *     Proposition 1).  L = T*H*W.
+ *   - A mask block (the paper's PSABlock) is a brick of tile.bt x tile.bh x tile.bw
+ *     tokens.  Block grid T' = ceil(T/bt), H' = ceil(H/bh), W' = ceil(W/bw),
+ *     S' = H'*W', NB = T'*S'.  Block id = t'*S' + h'*W' + w'.
+ *   - The six parameters are in block units.  Query block (t'_q, s'_q) attends key
+ *     block (t'_k, s'_k) iff  (|t'_k - t'_q - T_o| mod T_s) <= T_w - 1  and
+ *     (|s'_k - s'_q - S_o| mod S_s) <= S_w - 1  (Algorithm 1).  A stride of 0 encodes
+ *     an infinite stride: no modulo, one diagonal band (Appendix C.2).
+ *   - "host" / "device" on a pointer says where the memory must live.  The library
+ *     never takes ownership of caller memory.  Device work is enqueued on `stream`
+ *     (a cudaStream_t passed as void*; NULL = the default stream) and the calls
+ *     return without synchronising unless stated.
+ *   - Return value: PSA_OK (0) or a negative psa_status.  Nothing is thrown, printed
+ *     or aborted.
+ *   - The library keeps one lazily created device workspace per device (work order,
+ *     status word); calls that overlap on the GPU from different streams race on it.
+ *     psa_shutdown() frees it.
+ */
+#ifndef PSA_H_
+#define PSA_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  PSA_OK = 0,
+  PSA_ERR_INVALID_ARG = -1, /* null/misaligned pointer, non-positive extent, bad parameter   */
+  PSA_ERR_UNSUPPORTED = -2, /* head_dim != 128, tile token count not 128/256/384, not sm_100  */
+  PSA_ERR_CAPACITY = -3,    /* col_capacity < nnz                                             */
+  PSA_ERR_CUDA = -4,        /* a CUDA runtime/driver call failed                              */
+  PSA_ERR_TIMEOUT = -5      /* a bounded device-side wait expired (see psa_last_device_status) */
+} psa_status;
+
+/* Six stripe parameters of one head, in block units (Section 3.2).  Ts == 0 / Ss == 0
+ * mean an infinite stride.  Valid: Tw, Sw >= 1; Ts, Ss >= 0; |To|, |So| < 2^30. */
+typedef struct { int32_t Tw, To, Ts, Sw, So, Ss; } psa_head_params;
+
+/* Mask block (PSABlock) extents in tokens.  For psa_attn_fwd bt*bh*bw must be 128, 256
+ * or 384 and split into 128-token slabs along its outermost non-unit axis. */
+typedef struct { int32_t bt, bh, bw; } psa_tile;
+
+typedef struct {
+  int32_t  n_heads;      /* >= 1                                                          */
+  int32_t  head_dim;     /* must be 128 for psa_attn_fwd                                   */
+  psa_tile tile;
+  float    scale;        /* softmax scale applied to q.k (the configs use 1/sqrt(128))     */
+  int64_t  stride_head;  /* elements between heads, shared by q, k, v, out                 */
+  int64_t  stride_token; /* elements between tokens (>= head_dim, multiple of 8)           */
+} psa_problem;
+
+/* Sizes of psa_mask_build's outputs.  *nb = NB; *nnz = number of attended block pairs
+ * summed over heads (exact; params is host memory, n_heads entries).  Pure host code. */
+int psa_mask_sizes(const psa_head_params* params, const psa_problem* prob,
+                   int T, int H, int W, int64_t* nb, int64_t* nnz);
+
+/* GetKVBlocks for every (head, query block) (Algorithm 2, producer; Algorithm 1):
+ *   block_mask  device uint8 [n_heads][NB][NB], 1 = attended (row = query block)
+ *   row_ptr     device int32 [n_heads*NB + 1], exclusive prefix sum of row counts in
+ *               (head, query block) order
+ *   col_idx     device int32 [col_capacity], ascending key-block ids of each row
+ * params: host, n_heads entries.  If col_capacity < nnz nothing is launched and
+ * PSA_ERR_CAPACITY is returned (use psa_mask_sizes).  Any of the three outputs may be
+ * NULL to skip it (col_idx needs row_ptr).  Integer work only; results are exact. */
+int psa_mask_build(const psa_head_params* params, const psa_problem* prob,
+                   int T, int H, int W, uint8_t* block_mask, int32_t* row_ptr,
+                   int32_t* col_idx, int64_t col_capacity, void* stream);
+
+/* Forward pass (Algorithm 2 with the mask of Algorithm 1 decided in-kernel):
+ *   q, k, v   device bf16, element (head, token, c) at head*stride_head + token*stride_token + c
+ *   out       device bf16, same strides; must not alias the inputs
+ *   lse       device fp32 [n_heads][L], natural log of the sum of exp(scale * q.k) over
+ *             attended real keys
+ *   head_params host, n_heads entries
+ * Rows whose query block attends no key block get out = 0 and lse = -inf.  Padded
+ * positions (Section 3.2, "3D-Padding") are never read from or written to memory.
+ * Pointers must be 16-byte aligned.  bf16 inputs, fp32 accumulation. */
+int psa_attn_fwd(const void* q, const void* k, const void* v, void* out, float* lse,
+                 const psa_head_params* head_params, const psa_problem* prob,
+                 int T, int H, int W, void* stream);
+
+/* The same call for HOST tensors: copies q, k, v (host, pinned for speed) into the
+ * caller's device staging buffers d_q, d_k, d_v, runs psa_attn_fwd into d_out / d_lse
+ * and copies the results to out / lse (host), all on `stream`, then synchronises it.
+ * Each staging buffer must hold the full strided extent of its tensor:
+ * (n_heads-1)*stride_head + (L-1)*stride_token + head_dim elements. */
+int psa_attn_fwd_host(const void* q, const void* k, const void* v, void* out, float* lse,
+                      void* d_q, void* d_k, void* d_v, void* d_out, float* d_lse,
+                      const psa_head_params* head_params, const psa_problem* prob,
+                      int T, int H, int W, void* stream);
+
+/* Synchronises the current device, then returns the status word the last psa_attn_fwd
+ * on it left behind: PSA_OK, or PSA_ERR_TIMEOUT if a bounded wait inside the kernel
+ * expired (outputs are then undefined).  *detail (optional, host) receives a
+ * diagnostic code naming the wait that gave up. */
+int psa_last_device_status(int32_t* detail);
+
+/* Number of kernels the library has launched since load (all entry points). */
+int64_t psa_launch_count(void);
+
+/* Frees the per-device workspaces.  Safe to call more than once. */
+int psa_shutdown(void);
+
+const char* psa_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PSA_H_ */

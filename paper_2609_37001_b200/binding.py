@@ -1,0 +1,200 @@
+"""Thin ctypes binding of libpsa.so: argument marshalling only.
+
+Every step of the path runs inside the CUDA library; torch is used for device memory
+and streams.  Importing this module without a built library, or calling it without a
+CUDA device, raises -- there is no CPU fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence, Tuple
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libpsa.so")
+
+PSA_OK = 0
+PSA_ERR_INVALID_ARG = -1
+PSA_ERR_UNSUPPORTED = -2
+PSA_ERR_CAPACITY = -3
+PSA_ERR_CUDA = -4
+PSA_ERR_TIMEOUT = -5
+
+
+class PsaError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        super().__init__(f"{what}: {status_string(status)} ({status})")
+
+
+class HeadParams(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in ("Tw", "To", "Ts", "Sw", "So", "Ss")]
+
+
+class Tile(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in ("bt", "bh", "bw")]
+
+
+class Problem(ctypes.Structure):
+    _fields_ = [("n_heads", ctypes.c_int32), ("head_dim", ctypes.c_int32), ("tile", Tile),
+                ("scale", ctypes.c_float), ("stride_head", ctypes.c_int64), ("stride_token", ctypes.c_int64)]
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libpsa.so (built by paper_2609_37001_b200.build); raises if it is missing."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: run `python -m paper_2609_37001_b200.build`")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i32, i64p = ctypes.c_void_p, ctypes.c_int, ctypes.POINTER(ctypes.c_int64)
+        hp, pp = ctypes.POINTER(HeadParams), ctypes.POINTER(Problem)
+        L.psa_status_string.restype = ctypes.c_char_p
+        L.psa_status_string.argtypes = [i32]
+        L.psa_launch_count.restype = ctypes.c_int64
+        L.psa_launch_count.argtypes = []
+        L.psa_mask_sizes.argtypes = [hp, pp, i32, i32, i32, i64p, i64p]
+        L.psa_mask_build.argtypes = [hp, pp, i32, i32, i32, vp, vp, vp, ctypes.c_int64, vp]
+        L.psa_attn_fwd.argtypes = [vp, vp, vp, vp, vp, hp, pp, i32, i32, i32, vp]
+        L.psa_attn_fwd_host.argtypes = [vp] * 10 + [hp, pp, i32, i32, i32, vp]
+        L.psa_last_device_status.argtypes = [ctypes.POINTER(ctypes.c_int32)]
+        L.psa_shutdown.argtypes = []
+        for f in (L.psa_mask_sizes, L.psa_mask_build, L.psa_attn_fwd, L.psa_attn_fwd_host,
+                  L.psa_last_device_status, L.psa_shutdown):
+            f.restype = ctypes.c_int
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().psa_status_string(int(status)).decode()
+
+
+def _check(status: int, what: str) -> None:
+    if status != PSA_OK:
+        raise PsaError(status, what)
+
+
+def _params_array(head_params: Sequence[Sequence[int]]):
+    arr = (HeadParams * len(head_params))()
+    for i, p in enumerate(head_params):
+        arr[i] = HeadParams(*[int(x) for x in p])
+    return arr
+
+
+def make_problem(n_heads: int, tile: Sequence[int], scale: float, stride_head: int, stride_token: int,
+                 head_dim: int = 128) -> Problem:
+    return Problem(int(n_heads), int(head_dim), Tile(*[int(x) for x in tile]), float(scale),
+                   int(stride_head), int(stride_token))
+
+
+def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return int(s.cuda_stream)
+
+
+def _require_cuda(*tensors: torch.Tensor) -> None:
+    for t in tensors:
+        if not t.is_cuda:
+            raise ValueError("device tensors required")
+
+
+def psa_mask_sizes(head_params, grid: Sequence[int], tile: Sequence[int]) -> Tuple[int, int]:
+    """(NB, nnz) for psa_mask_build's outputs.  Host arithmetic only."""
+    prob = make_problem(len(head_params), tile, 1.0, 0, 128)
+    nb, nnz = ctypes.c_int64(0), ctypes.c_int64(0)
+    T, H, W = (int(x) for x in grid)
+    _check(lib().psa_mask_sizes(_params_array(head_params), ctypes.byref(prob), T, H, W,
+                                ctypes.byref(nb), ctypes.byref(nnz)), "psa_mask_sizes")
+    return nb.value, nnz.value
+
+
+def psa_mask_build(head_params, grid: Sequence[int], tile: Sequence[int], device="cuda",
+                   out: Optional[Tuple[torch.Tensor, torch.Tensor, torch.Tensor]] = None,
+                   stream: Optional[torch.cuda.Stream] = None):
+    """Block mask uint8[heads, NB, NB], row_ptr int32[heads*NB+1], col_idx int32[nnz] on the device."""
+    nh = len(head_params)
+    T, H, W = (int(x) for x in grid)
+    if out is None:
+        nb, nnz = psa_mask_sizes(head_params, grid, tile)
+        mask = torch.empty((nh, nb, nb), dtype=torch.uint8, device=device)
+        row_ptr = torch.empty(nh * nb + 1, dtype=torch.int32, device=device)
+        col_idx = torch.empty(max(nnz, 1), dtype=torch.int32, device=device)
+    else:
+        mask, row_ptr, col_idx = out
+        nnz = None
+    _require_cuda(mask, row_ptr, col_idx)
+    prob = make_problem(nh, tile, 1.0, 0, 128)
+    _check(lib().psa_mask_build(_params_array(head_params), ctypes.byref(prob), T, H, W, mask.data_ptr(),
+                                row_ptr.data_ptr(), col_idx.data_ptr(), col_idx.numel(), _stream_ptr(stream)),
+           "psa_mask_build")
+    if nnz is not None:
+        col_idx = col_idx[:nnz]
+    return mask, row_ptr, col_idx
+
+
+def psa_attn_fwd(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, head_params, grid: Sequence[int],
+                 tile: Sequence[int], scale: float, out: Optional[torch.Tensor] = None,
+                 lse: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None):
+    """q, k, v: bf16 device tensors [heads, L, 128] (any head/token strides, last dim contiguous,
+    shared by all three).  Returns (out bf16 like q, lse fp32 [heads, L])."""
+    _require_cuda(q, k, v)
+    if q.dtype != torch.bfloat16 or k.dtype != torch.bfloat16 or v.dtype != torch.bfloat16:
+        raise ValueError("bf16 tensors required")
+    nh, L, d = q.shape
+    T, H, W = (int(x) for x in grid)
+    if L != T * H * W or k.shape != q.shape or v.shape != q.shape:
+        raise ValueError("shape mismatch")
+    if q.stride() != k.stride() or q.stride() != v.stride() or q.stride(2) != 1:
+        raise ValueError("q, k, v must share strides with a contiguous last dimension")
+    if out is None:
+        out = torch.empty_strided(q.shape, q.stride(), dtype=q.dtype, device=q.device)
+    if lse is None:
+        lse = torch.empty((nh, L), dtype=torch.float32, device=q.device)
+    if out.stride() != q.stride() or not lse.is_contiguous():
+        raise ValueError("out must share q's strides; lse must be contiguous")
+    prob = make_problem(nh, tile, scale, q.stride(0), q.stride(1), d)
+    _check(lib().psa_attn_fwd(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), lse.data_ptr(),
+                              _params_array(head_params), ctypes.byref(prob), T, H, W, _stream_ptr(stream)),
+           "psa_attn_fwd")
+    return out, lse
+
+
+def psa_attn_fwd_host(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, out: torch.Tensor, lse: torch.Tensor,
+                      staging: Sequence[torch.Tensor], head_params, grid: Sequence[int], tile: Sequence[int],
+                      scale: float, stream: Optional[torch.cuda.Stream] = None) -> None:
+    """Host-tensor variant: q, k, v, out (bf16 [heads, L, 128], contiguous) and lse (fp32 [heads, L])
+    live in host memory; ``staging`` = (d_q, d_k, d_v, d_out, d_lse) are device buffers of the same
+    shapes.  Copies in, runs, copies out and synchronises the stream."""
+    d_q, d_k, d_v, d_out, d_lse = staging
+    _require_cuda(d_q, d_k, d_v, d_out, d_lse)
+    for t in (q, k, v, out, lse):
+        if t.is_cuda or not t.is_contiguous():
+            raise ValueError("contiguous host tensors required")
+    nh, L, d = q.shape
+    T, H, W = (int(x) for x in grid)
+    prob = make_problem(nh, tile, scale, q.stride(0), q.stride(1), d)
+    _check(lib().psa_attn_fwd_host(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), lse.data_ptr(),
+                                   d_q.data_ptr(), d_k.data_ptr(), d_v.data_ptr(), d_out.data_ptr(),
+                                   d_lse.data_ptr(), _params_array(head_params), ctypes.byref(prob), T, H, W,
+                                   _stream_ptr(stream)), "psa_attn_fwd_host")
+
+
+def psa_last_device_status() -> Tuple[int, int]:
+    """Synchronises the device; returns (status, detail) left by the last psa_attn_fwd."""
+    detail = ctypes.c_int32(0)
+    st = lib().psa_last_device_status(ctypes.byref(detail))
+    return st, detail.value
+
+
+def psa_launch_count() -> int:
+    return int(lib().psa_launch_count())
+
+
+def psa_shutdown() -> None:
+    _check(lib().psa_shutdown(), "psa_shutdown")

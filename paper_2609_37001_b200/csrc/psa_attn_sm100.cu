@@ -1,0 +1,709 @@
+// psa_attn_fwd for sm_100a: stripe-masked flash attention forward.
+//
+// One persistent CTA per SM walks a list of work items ordered by the number of
+// attended key blocks.  A work item is up to two 128-row query slabs of one query
+// block (PSABlock); both slabs share the block's key list (GetKVBlocks, Algorithm 2),
+// which the load warp enumerates in ascending block id straight from the six stripe
+// parameters (Algorithm 1) -- no mask or index list is read from memory.
+//
+// Roles (320 threads):
+//   warps 0-3  softmax / correction / epilogue of query slab 0  (TMEM lanes 0..127)
+//   warps 4-7  the same for query slab 1
+//   warp  8    TMA loads: Q slabs once per item, K and V slabs through a 5-slot ring
+//   warp  9    tcgen05.mma issue: S_i = Q_i K^T (SS form), O_i += P_i V (P read from TMEM)
+// TMEM (512 columns): S0 | S1 | O0 | O1, 128 fp32 columns each; the bf16 probabilities
+// P_i overwrite the first 64 columns of S_i.
+// Every wait is bounded; on expiry the CTA records a status word and unwinds.
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include "psa_common.cuh"
+
+namespace psa {
+
+constexpr int kThreads = 320;
+constexpr int kNumSlots = 5;                       // K/V ring slots of one 128 x 128 bf16 slab
+constexpr uint32_t kSlabBytes = 128 * 128 * 2;     // 32 KB
+constexpr uint32_t kHalfBytes = kSlabBytes / 2;    // one 64-column swizzled half
+constexpr int kMetaRing = 8;
+constexpr float kRescaleThreshold = 8.0f;          // log2 units; lazy rescale of O
+constexpr unsigned long long kTimeoutNs = 2000000000ull;
+
+// shared memory map (offsets from a 1024-byte aligned base)
+constexpr uint32_t kOffQ = 0;                                   // 2 slabs
+constexpr uint32_t kOffRing = 2 * kSlabBytes;                   // kNumSlots slabs
+constexpr uint32_t kOffBar = kOffRing + kNumSlots * kSlabBytes; // mbarriers
+constexpr int kBarQFull = 0, kBarQEmpty = 2, kBarSlotFull = 4, kBarSlotEmpty = 4 + kNumSlots,
+              kBarSFull = 4 + 2 * kNumSlots, kBarPReady = kBarSFull + 2, kBarOFull = kBarPReady + 2,
+              kBarOEmpty = kBarOFull + 2, kNumBars = kBarOEmpty + 2;
+constexpr uint32_t kOffMeta = kOffBar + kNumBars * 8;           // kMetaRing x 8 words
+constexpr uint32_t kOffMaskT = kOffMeta + kMetaRing * 32;       // kMaxTp / 32 words
+constexpr uint32_t kOffMaskS = kOffMaskT + (kMaxTp / 32) * 4;   // kMaxSp / 32 words
+constexpr uint32_t kOffMisc = kOffMaskS + (kMaxSp / 32) * 4;    // tmem base, abort flag
+constexpr uint32_t kSmemBytes = kOffMisc + 16;
+constexpr uint32_t kSmemAlloc = kSmemBytes + 1024;              // slack for manual alignment
+
+// ----------------------------------------------------------------------------- PTX
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ unsigned long long globaltimer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait.  Returns false once the CTA-wide abort flag is set (by this or another
+// waiter); `code` names the wait for the status word.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int code) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = globaltimer_ns();
+  uint32_t n = 0;
+  while (!mbar_try_wait(bar, parity)) {
+    if ((++n & 255u) == 0u) {
+      if (*abort_flag != 0) return false;
+      if (globaltimer_ns() - t0 > kTimeoutNs) {
+        atomicCAS((int*)abort_flag, 0, code);
+        return false;
+      }
+    }
+  }
+  return true;
+}
+// warp-uniform variant: every lane waits, the warp agrees on the outcome
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag, int code) {
+  const bool ok = mbar_wait(bar, parity, abort_flag, code);
+  return __all_sync(0xffffffffu, ok);
+}
+
+__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* tm, uint32_t bar,
+                                            int c0, int c1, int c2, int c3, int c4) {
+  asm volatile(
+      "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+      ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4) : "memory");
+}
+__device__ __forceinline__ void tma_store_5d(const CUtensorMap* tm, uint32_t src,
+                                             int c0, int c1, int c2, int c3, int c4) {
+  asm volatile(
+      "cp.async.bulk.tensor.5d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5, %6}], [%1];"
+      ::"l"(tm), "r"(src), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4) : "memory");
+}
+__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[smem desc] * B[smem desc]
+__device__ __forceinline__ void tc_mma_ss(uint32_t d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem desc]
+__device__ __forceinline__ void tc_mma_ts(uint32_t d, uint32_t a, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(d), "r"(a), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t addr, float* v) {
+  uint32_t* r = reinterpret_cast<uint32_t*>(v);
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(addr) : "memory");
+}
+__device__ __forceinline__ void tc_st32(uint32_t addr, const float* v) {
+  const uint32_t* r = reinterpret_cast<const uint32_t*>(v);
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+      ::"r"(addr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+        "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+        "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+__device__ __forceinline__ void tc_st16(uint32_t addr, const uint32_t* r) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+      ::"r"(addr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+      : "memory");
+}
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+__device__ __forceinline__ void named_bar_sync(int id, int nthreads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle, sm_100 version field.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr >> 4) & 0x3FFFu);
+  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+  d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+  d |= 1ull << 46;  // descriptor version
+  d |= 2ull << 61;  // 128-byte swizzle
+  return d;
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = 128; A is K-major.
+__host__ __device__ constexpr uint32_t instr_desc(bool b_mn_major) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+}
+
+// ----------------------------------------------------------------------------- planning
+// Work order: per head, query blocks ranked by attended key-block count (largest first),
+// heads kept together so that concurrently running CTAs share K/V in L2.
+__global__ void __launch_bounds__(256)
+plan_kernel(const HeadParamsArray hp, const Geom g, int head0, int* __restrict__ ws_header,
+            psa_head_params* __restrict__ hp_dev, WorkItem* __restrict__ items) {
+  extern __shared__ int sm[];  // cntT[Tp], cntS[Sp], cnt[NB]
+  int* cntT = sm;
+  int* cntS = sm + g.Tp;
+  int* cnt = cntS + g.Sp;
+  const int h = blockIdx.x;
+  const psa_head_params p = hp.p[head0 + h];
+  if (h == 0 && threadIdx.x < kWsHeaderWords) ws_header[threadIdx.x] = 0;
+  if (threadIdx.x == 0) hp_dev[h] = p;
+  for (int a = threadIdx.x; a < g.Tp + g.Sp; a += blockDim.x) {
+    int c = 0;
+    if (a < g.Tp) {
+      for (int k = 0; k < g.Tp; ++k) c += axis_attends(k - a, p.Tw, p.To, p.Ts);
+    } else {
+      for (int k = 0; k < g.Sp; ++k) c += axis_attends(k - (a - g.Tp), p.Sw, p.So, p.Ss);
+    }
+    sm[a] = c;
+  }
+  __syncthreads();
+  for (int qb = threadIdx.x; qb < g.NB; qb += blockDim.x) cnt[qb] = cntT[qb / g.Sp] * cntS[qb % g.Sp];
+  __syncthreads();
+  const int ipb = g.items_per_block;
+  WorkItem* out = items + (size_t)h * g.NB * ipb;
+  for (int qb = threadIdx.x; qb < g.NB; qb += blockDim.x) {
+    const int c = cnt[qb];
+    int rank = 0;
+    for (int j = 0; j < g.NB; ++j) {
+      const int cj = cnt[j];
+      rank += (cj > c) || (cj == c && j < qb);
+    }
+    // two-slab items first (heavier), then the odd single-slab items, each in rank order
+    int pos = rank;
+    for (int it = 0; it < ipb; ++it) {
+      const int sub0 = 2 * it;
+      const int nq = (g.n_sub - sub0) >= 2 ? 2 : 1;
+      out[(size_t)it * g.NB + pos] = make_int4(h, qb, c, sub0 | (nq << 16));
+    }
+  }
+}
+
+// ----------------------------------------------------------------------------- attention
+struct AttnParams {
+  Geom g;
+  const WorkItem* items;
+  const psa_head_params* hp_dev;
+  int* ws_header;
+  float* lse;     // already offset to the first head of this launch
+  int n_items;
+};
+
+__device__ __forceinline__ void slab_origin(const Geom& g, int qb, int sub, int& t0, int& h0, int& w0) {
+  const int tb = qb / g.Sp, sb = qb % g.Sp;
+  t0 = tb * g.bt;
+  h0 = (sb / g.Wp) * g.bh;
+  w0 = (sb % g.Wp) * g.bw;
+  if (g.sub_axis == 0) t0 += sub * g.ct;
+  else if (g.sub_axis == 1) h0 += sub * g.ch;
+  else w0 += sub * g.cw;
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o,
+                const AttnParams prm) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const uint32_t sbase = smem_u32(smem);
+  const Geom& g = prm.g;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  auto bar = [&](int idx) -> uint32_t { return sbase + kOffBar + 8u * (uint32_t)idx; };
+  uint32_t* meta = reinterpret_cast<uint32_t*>(smem + kOffMeta);
+  uint32_t* maskT = reinterpret_cast<uint32_t*>(smem + kOffMaskT);
+  uint32_t* maskS = reinterpret_cast<uint32_t*>(smem + kOffMaskS);
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + kOffMisc);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kOffMisc + 4);
+
+  if (threadIdx.x == 0) {
+    *abort_flag = 0;
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(bar(kBarQFull + i), 1);
+      mbar_init(bar(kBarQEmpty + i), 1);
+      mbar_init(bar(kBarSFull + i), 1);
+      mbar_init(bar(kBarPReady + i), 128);
+      mbar_init(bar(kBarOFull + i), 1);
+      mbar_init(bar(kBarOEmpty + i), 128);
+    }
+    for (int s = 0; s < kNumSlots; ++s) {
+      mbar_init(bar(kBarSlotFull + s), 1);
+      mbar_init(bar(kBarSlotEmpty + s), 1);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 9) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(sbase + kOffMisc), "r"(512) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+
+  if (warp == 8) {
+    // ======================================================================= load warp
+    uint32_t tile_g = 0;       // ring tiles issued so far (K and V alternate)
+    uint32_t kv_g = 0;         // key slabs issued so far
+    uint32_t it_q[2] = {0, 0}; // items in which query slab i was active
+    bool ok = true;
+    for (int idx = blockIdx.x; ok && idx < prm.n_items; idx += gridDim.x) {
+      const WorkItem wi = prm.items[idx];
+      const int head = wi.x, qb = wi.y, sub0 = wi.w & 0xffff, nq = wi.w >> 16;
+      const psa_head_params p = prm.hp_dev[head];
+      const int tq = qb / g.Sp, sq = qb % g.Sp;
+      // attended key-block coordinates of this query block, one bit per block coordinate
+      for (int b = 0; b < g.Tp; b += 32) {
+        const int tk = b + lane;
+        const unsigned m = __ballot_sync(0xffffffffu, tk < g.Tp && axis_attends(tk - tq, p.Tw, p.To, p.Ts));
+        if (lane == 0) maskT[b >> 5] = m;
+      }
+      for (int b = 0; b < g.Sp; b += 32) {
+        const int sk = b + lane;
+        const unsigned m = __ballot_sync(0xffffffffu, sk < g.Sp && axis_attends(sk - sq, p.Sw, p.So, p.Ss));
+        if (lane == 0) maskS[b >> 5] = m;
+      }
+      __syncwarp();
+      // query slabs
+      for (int i = 0; i < nq; ++i) {
+        ok = mbar_wait_warp(bar(kBarQEmpty + i), (it_q[i] & 1u) ^ 1u, abort_flag, 0x100 + i);
+        if (!ok) break;
+        if (lane == 0) {
+          int t0, h0, w0;
+          slab_origin(g, qb, sub0 + i, t0, h0, w0);
+          const uint32_t dst = sbase + kOffQ + (uint32_t)i * kSlabBytes;
+          mbar_expect_tx(bar(kBarQFull + i), kSlabBytes);
+          tma_load_5d(dst, &tm_q, bar(kBarQFull + i), 0, w0, h0, t0, head);
+          tma_load_5d(dst + kHalfBytes, &tm_q, bar(kBarQFull + i), 64, w0, h0, t0, head);
+        }
+        ++it_q[i];
+      }
+      if (!ok) break;
+      // key / value slabs in ascending key-block id
+      for (int tw = 0; ok && tw < g.Tp; tw += 32) {
+        uint32_t mt = maskT[tw >> 5];
+        while (ok && mt) {
+          const int tk = tw + __ffs(mt) - 1;
+          mt &= mt - 1;
+          for (int sw = 0; ok && sw < g.Sp; sw += 32) {
+            uint32_t ms = maskS[sw >> 5];
+            while (ok && ms) {
+              const int sk = sw + __ffs(ms) - 1;
+              ms &= ms - 1;
+              const int kb = tk * g.Sp + sk;
+              for (int sub = 0; ok && sub < g.n_sub; ++sub) {
+                int t0, h0, w0;
+                slab_origin(g, kb, sub, t0, h0, w0);
+                // validity of the slab's 128 key positions (3D-padding): bit c of word c/32
+                const bool edge = (t0 + g.ct > g.T) || (h0 + g.ch > g.H) || (w0 + g.cw > g.W);
+                uint32_t vw[4] = {0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu};
+                if (edge) {
+#pragma unroll
+                  for (int w4 = 0; w4 < 4; ++w4) {
+                    const int c = w4 * 32 + lane;
+                    const int wi_ = c % g.cw, hi_ = (c / g.cw) % g.ch, ti_ = c / (g.cw * g.ch);
+                    vw[w4] = __ballot_sync(0xffffffffu, (t0 + ti_ < g.T) && (h0 + hi_ < g.H) && (w0 + wi_ < g.W));
+                  }
+                }
+                const uint32_t sk_slot = tile_g % kNumSlots, sk_use = tile_g / kNumSlots;
+                ok = mbar_wait_warp(bar(kBarSlotEmpty + sk_slot), (sk_use & 1u) ^ 1u, abort_flag, 0x110);
+                if (!ok) break;
+                if (lane == 0) {
+                  uint32_t* m = meta + (kv_g % kMetaRing) * 8;
+                  m[0] = edge ? 1u : 0u;
+                  m[1] = vw[0]; m[2] = vw[1]; m[3] = vw[2]; m[4] = vw[3];
+                  const uint32_t dst = sbase + kOffRing + sk_slot * kSlabBytes;
+                  mbar_expect_tx(bar(kBarSlotFull + sk_slot), kSlabBytes);
+                  tma_load_5d(dst, &tm_k, bar(kBarSlotFull + sk_slot), 0, w0, h0, t0, head);
+                  tma_load_5d(dst + kHalfBytes, &tm_k, bar(kBarSlotFull + sk_slot), 64, w0, h0, t0, head);
+                }
+                ++tile_g;
+                const uint32_t sv_slot = tile_g % kNumSlots, sv_use = tile_g / kNumSlots;
+                ok = mbar_wait_warp(bar(kBarSlotEmpty + sv_slot), (sv_use & 1u) ^ 1u, abort_flag, 0x111);
+                if (!ok) break;
+                if (lane == 0) {
+                  const uint32_t dst = sbase + kOffRing + sv_slot * kSlabBytes;
+                  mbar_expect_tx(bar(kBarSlotFull + sv_slot), kSlabBytes);
+                  tma_load_5d(dst, &tm_v, bar(kBarSlotFull + sv_slot), 0, w0, h0, t0, head);
+                  tma_load_5d(dst + kHalfBytes, &tm_v, bar(kBarSlotFull + sv_slot), 64, w0, h0, t0, head);
+                }
+                ++tile_g;
+                ++kv_g;
+              }
+            }
+          }
+        }
+      }
+    }
+    // Let every load that was issued land before the CTA retires: wait for each slot's
+    // last issued phase (bounded; the abort flag no longer cuts these short).
+    if (lane == 0) {
+      for (uint32_t back = 0; back < (uint32_t)kNumSlots && back < tile_g; ++back) {
+        const uint32_t tg = tile_g - 1 - back;
+        const uint32_t slot = tg % kNumSlots, use = tg / kNumSlots;
+        const unsigned long long t0 = globaltimer_ns();
+        while (!mbar_try_wait(bar(kBarSlotFull + slot), use & 1u)) {
+          if (globaltimer_ns() - t0 > kTimeoutNs) break;
+        }
+      }
+      for (int i = 0; i < 2; ++i) {
+        if (it_q[i] == 0) continue;
+        const unsigned long long t0 = globaltimer_ns();
+        while (!mbar_try_wait(bar(kBarQFull + i), (it_q[i] - 1) & 1u)) {
+          if (globaltimer_ns() - t0 > kTimeoutNs) break;
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 9) {
+    // ======================================================================= MMA warp
+    constexpr uint32_t kIdescQK = instr_desc(false);
+    constexpr uint32_t kIdescPV = instr_desc(true);
+    uint32_t tile_g = 0;
+    uint32_t it_q[2] = {0, 0};
+    uint32_t cnt_s[2] = {0, 0};  // S_i tiles produced; P_i tiles consumed so far
+    bool ok = true;
+
+    // S_i = Q_i K^T over head_dim = 128: 8 MMAs of K = 16; both operands K-major, SW128.
+    auto issue_qk = [&](int i, uint32_t kslot) {
+      const uint32_t qaddr = sbase + kOffQ + (uint32_t)i * kSlabBytes;
+      const uint32_t kaddr = sbase + kOffRing + kslot * kSlabBytes;
+#pragma unroll
+      for (int kk = 0; kk < 8; ++kk) {
+        const uint32_t off = (uint32_t)(kk >> 2) * kHalfBytes + (uint32_t)(kk & 3) * 32u;
+        tc_mma_ss(tmem + (uint32_t)i * 128u, smem_desc(qaddr + off, 16, 1024), smem_desc(kaddr + off, 16, 1024),
+                  kIdescQK, kk > 0 ? 1u : 0u);
+      }
+    };
+    // O_i (+)= P_i V over 128 keys: 8 MMAs of K = 16; A = bf16 P in TMEM (8 columns per
+    // step), B = V slab as loaded (keys x head_dim, head_dim contiguous) = MN-major SW128:
+    // 16 keys advance 2048 bytes, the second 64 columns of head_dim sit one half further.
+    auto issue_pv = [&](int i, uint32_t vslot, bool accumulate) {
+      const uint32_t vaddr = sbase + kOffRing + vslot * kSlabBytes;
+#pragma unroll
+      for (int kk = 0; kk < 8; ++kk) {
+        tc_mma_ts(tmem + 256u + (uint32_t)i * 128u, tmem + (uint32_t)i * 128u + (uint32_t)kk * 8u,
+                  smem_desc(vaddr + (uint32_t)kk * 2048u, kHalfBytes, 1024), kIdescPV,
+                  (accumulate || kk > 0) ? 1u : 0u);
+      }
+    };
+
+    for (int idx = blockIdx.x; ok && idx < prm.n_items; idx += gridDim.x) {
+      const WorkItem wi = prm.items[idx];
+      const int nq = wi.w >> 16;
+      const int n_kv = wi.z * g.n_sub;
+      for (int i = 0; i < nq; ++i) {
+        ok = mbar_wait_warp(bar(kBarQFull + i), it_q[i] & 1u, abort_flag, 0x200 + i);
+        if (!ok) break;
+        // the epilogue of the previous item must have drained O_i before it is overwritten
+        ok = mbar_wait_warp(bar(kBarOEmpty + i), (it_q[i] & 1u) ^ 1u, abort_flag, 0x202 + i);
+        if (!ok) break;
+      }
+      if (!ok) break;
+      if (n_kv > 0) {
+        // first key slab: both S tiles
+        {
+          const uint32_t slot = tile_g % kNumSlots, use = tile_g / kNumSlots;
+          ok = mbar_wait_warp(bar(kBarSlotFull + slot), use & 1u, abort_flag, 0x210);
+          if (!ok) break;
+          tc_fence_after();
+          if (lane == 0) {
+            for (int i = 0; i < nq; ++i) {
+              issue_qk(i, slot);
+              tc_commit(bar(kBarSFull + i));
+            }
+            tc_commit(bar(kBarSlotEmpty + slot));
+          }
+          __syncwarp();
+          ++tile_g;
+        }
+        for (int j = 0; ok && j < n_kv; ++j) {
+          const uint32_t vslot = tile_g % kNumSlots, vuse = tile_g / kNumSlots;
+          ok = mbar_wait_warp(bar(kBarSlotFull + vslot), vuse & 1u, abort_flag, 0x211);
+          if (!ok) break;
+          ++tile_g;
+          const bool more = (j + 1 < n_kv);
+          uint32_t kslot = 0;
+          if (more) {
+            kslot = tile_g % kNumSlots;
+            const uint32_t kuse = tile_g / kNumSlots;
+            ok = mbar_wait_warp(bar(kBarSlotFull + kslot), kuse & 1u, abort_flag, 0x212);
+            if (!ok) break;
+            ++tile_g;
+          }
+          for (int i = 0; ok && i < nq; ++i) {
+            ok = mbar_wait_warp(bar(kBarPReady + i), cnt_s[i] & 1u, abort_flag, 0x220 + i);
+            if (!ok) break;
+            ++cnt_s[i];
+            tc_fence_after();
+            if (lane == 0) {
+              issue_pv(i, vslot, j > 0);
+              if (i == nq - 1) tc_commit(bar(kBarSlotEmpty + vslot));
+              if (more) {
+                issue_qk(i, kslot);
+                tc_commit(bar(kBarSFull + i));
+                if (i == nq - 1) tc_commit(bar(kBarSlotEmpty + kslot));
+              } else {
+                tc_commit(bar(kBarOFull + i));
+              }
+            }
+            __syncwarp();
+          }
+        }
+        if (!ok) break;
+      } else {
+        if (lane == 0) {
+          for (int i = 0; i < nq; ++i) tc_commit(bar(kBarOFull + i));
+        }
+        __syncwarp();
+      }
+      for (int i = 0; i < nq; ++i) ++it_q[i];
+    }
+  } else {
+    // ======================================================================= softmax warps
+    const int qi = warp >> 2;                     // query slab handled by this warpgroup
+    const int row = (warp & 3) * 32 + lane;       // row of the slab == TMEM lane
+    const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
+    const uint32_t tS = tmem + lane_addr + (uint32_t)qi * 128u;
+    const uint32_t tO = tmem + lane_addr + 256u + (uint32_t)qi * 128u;
+    uint32_t it_q = 0, cnt_s = 0, kv_g = 0;
+    bool ok = true;
+    const float neg_inf = __int_as_float(0xff800000);
+
+    for (int idx = blockIdx.x; ok && idx < prm.n_items; idx += gridDim.x) {
+      const WorkItem wi = prm.items[idx];
+      const int head = wi.x, qb = wi.y, sub0 = wi.w & 0xffff, nq = wi.w >> 16;
+      const int n_kv = wi.z * g.n_sub;
+      if (qi >= nq) {
+        kv_g += (uint32_t)n_kv;
+        continue;
+      }
+      float m_ref = neg_inf;  // running reference maximum, scaled log2 domain
+      float l = 0.f;          // running sum of exp2(s - m_ref)
+      for (int j = 0; ok && j < n_kv; ++j, ++kv_g) {
+        ok = mbar_wait_warp(bar(kBarSFull + qi), cnt_s & 1u, abort_flag, 0x300 + qi);
+        if (!ok) break;
+        ++cnt_s;
+        tc_fence_after();
+        float s[128];
+        tc_ld32(tS + 0, s + 0);
+        tc_ld32(tS + 32, s + 32);
+        tc_ld32(tS + 64, s + 64);
+        tc_ld32(tS + 96, s + 96);
+        tc_wait_ld();
+        const uint32_t* m = meta + (kv_g % kMetaRing) * 8;
+        if (m[0] != 0u) {  // 3D-padding: padded key positions score -inf
+          const uint32_t v0 = m[1], v1 = m[2], v2 = m[3], v3 = m[4];
+#pragma unroll
+          for (int c = 0; c < 32; ++c) {
+            if (!((v0 >> c) & 1u)) s[c] = neg_inf;
+            if (!((v1 >> c) & 1u)) s[32 + c] = neg_inf;
+            if (!((v2 >> c) & 1u)) s[64 + c] = neg_inf;
+            if (!((v3 >> c) & 1u)) s[96 + c] = neg_inf;
+          }
+        }
+        float mx = s[0];
+#pragma unroll
+        for (int c = 1; c < 128; ++c) mx = fmaxf(mx, s[c]);
+        const float ms = mx * g.scale_log2;
+        // Lazy rescale: the reference maximum only moves when the new maximum exceeds
+        // it by more than the threshold, so exponentials stay below 2^threshold.
+        float alpha = 1.f;
+        const bool grow = ms > m_ref + kRescaleThreshold;  // also true when m_ref == -inf
+        if (grow) {
+          alpha = fast_exp2(m_ref - ms);  // 0 when m_ref == -inf
+          m_ref = ms;
+        }
+        if (j > 0 && __any_sync(0xffffffffu, grow)) {
+          l *= alpha;
+#pragma unroll
+          for (int c4 = 0; c4 < 4; ++c4) {
+            float o[32];
+            tc_ld32(tO + c4 * 32, o);
+            tc_wait_ld();
+#pragma unroll
+            for (int c = 0; c < 32; ++c) o[c] *= alpha;
+            tc_st32(tO + c4 * 32, o);
+          }
+        }
+        const float m_use = (m_ref == neg_inf) ? 0.f : m_ref;
+        float sum = 0.f;
+#pragma unroll
+        for (int c4 = 0; c4 < 4; ++c4) {
+          uint32_t pk[16];
+#pragma unroll
+          for (int c = 0; c < 16; ++c) {
+            const float p0 = fast_exp2(fmaf(s[c4 * 32 + 2 * c], g.scale_log2, -m_use));
+            const float p1 = fast_exp2(fmaf(s[c4 * 32 + 2 * c + 1], g.scale_log2, -m_use));
+            sum += p0 + p1;
+            pk[c] = pack_bf16(p0, p1);
+          }
+          tc_st16(tS + c4 * 16, pk);
+        }
+        l += sum;
+        tc_wait_st();
+        tc_fence_before();
+        mbar_arrive(bar(kBarPReady + qi));
+      }
+      if (!ok) break;
+      // ---- epilogue: out = O / l, lse = ln2 * (m_ref + log2 l)
+      ok = mbar_wait_warp(bar(kBarOFull + qi), it_q & 1u, abort_flag, 0x310 + qi);
+      if (!ok) break;
+      ++it_q;
+      tc_fence_after();
+      const bool empty = (n_kv == 0) || !(l > 0.f);
+      const float inv = empty ? 0.f : 1.f / l;
+      uint8_t* stage = smem + kOffQ + (uint32_t)qi * kSlabBytes;
+#pragma unroll
+      for (int c4 = 0; c4 < 4; ++c4) {
+        float o[32];
+        if (n_kv > 0) {
+          tc_ld32(tO + c4 * 32, o);
+          tc_wait_ld();
+        }
+#pragma unroll
+        for (int c8 = 0; c8 < 4; ++c8) {
+          uint32_t w[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const float a = empty ? 0.f : o[c8 * 8 + 2 * e] * inv;
+            const float b = empty ? 0.f : o[c8 * 8 + 2 * e + 1] * inv;
+            w[e] = pack_bf16(a, b);
+          }
+          // 128-byte swizzle of the staging slab: 16-byte chunk index xor (row mod 8)
+          const int col = c4 * 32 + c8 * 8;
+          const int half = col >> 6, chunk = (col & 63) >> 3;
+          uint8_t* dst = stage + half * kHalfBytes + row * 128 + ((chunk ^ (row & 7)) << 4);
+          *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(bar(kBarOEmpty + qi));
+      int t0, h0, w0;
+      slab_origin(g, qb, sub0 + qi, t0, h0, w0);
+      {
+        const int wi_ = row % g.cw, hi_ = (row / g.cw) % g.ch, ti_ = row / (g.cw * g.ch);
+        const int t = t0 + ti_, hh = h0 + hi_, ww = w0 + wi_;
+        if (t < g.T && hh < g.H && ww < g.W) {
+          const long long tok = ((long long)t * g.H + hh) * g.W + ww;
+          prm.lse[(long long)head * g.L + tok] = empty ? neg_inf : (m_ref + log2f(l)) * 0.6931471805599453f;
+        }
+      }
+      fence_async_smem();
+      named_bar_sync(1 + qi, 128);
+      if ((warp & 3) == 0 && lane == 0) {
+        const uint32_t src = sbase + kOffQ + (uint32_t)qi * kSlabBytes;
+        tma_store_5d(&tm_o, src, 0, w0, h0, t0, head);
+        tma_store_5d(&tm_o, src + kHalfBytes, 64, w0, h0, t0, head);
+        tma_store_commit();
+        tma_store_wait_read();
+        mbar_arrive(bar(kBarQEmpty + qi));
+      }
+    }
+    if ((warp & 3) == 0 && lane == 0) tma_store_wait_all();
+  }
+
+  // ------------------------------------------------------------------------- teardown
+  tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x == 0 && *abort_flag != 0) {
+    if (atomicCAS(prm.ws_header + kWsStatus, 0, (int)PSA_ERR_TIMEOUT) == 0) prm.ws_header[kWsDetail] = *abort_flag;
+  }
+  if (warp == 9) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512) : "memory");
+  }
+}
+
+// ----------------------------------------------------------------------------- launchers
+size_t plan_smem_bytes(const Geom& g) { return sizeof(int) * (size_t)(g.Tp + g.Sp + g.NB); }
+
+cudaError_t launch_plan(const HeadParamsArray& hp, const Geom& g, int head0, int n_heads_here, int* ws_header,
+                        psa_head_params* hp_dev, WorkItem* items, cudaStream_t stream) {
+  const size_t smem = plan_smem_bytes(g);
+  if (smem > 48 * 1024) {
+    cudaError_t e = cudaFuncSetAttribute(plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+  }
+  plan_kernel<<<n_heads_here, 256, smem, stream>>>(hp, g, head0, ws_header, hp_dev, items);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_attn(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to,
+                        const Geom& g, const WorkItem* items, const psa_head_params* hp_dev, int* ws_header,
+                        float* lse, int n_items, int n_sms, cudaStream_t stream) {
+  {  // per device, cheap: set on every call
+    cudaError_t e = cudaFuncSetAttribute(attn_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemAlloc);
+    if (e != cudaSuccess) return e;
+  }
+  AttnParams prm;
+  prm.g = g;
+  prm.items = items;
+  prm.hp_dev = hp_dev;
+  prm.ws_header = ws_header;
+  prm.lse = lse;
+  prm.n_items = n_items;
+  const int grid = n_items < n_sms ? n_items : n_sms;
+  if (grid <= 0) return cudaSuccess;
+  attn_fwd_kernel<<<grid, kThreads, kSmemAlloc, stream>>>(tq, tk, tv, to, prm);
+  return cudaGetLastError();
+}
+
+}  // namespace psa

@@ -1,0 +1,54 @@
+// Shared host/device definitions of the PSA library (not part of the public ABI).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "psa.h"
+
+namespace psa {
+
+constexpr int kHeadDim = 128;     // head dimension the attention kernel is built for
+constexpr int kSlabTokens = 128;  // tokens per compute slab (one MMA tile of rows / keys)
+constexpr int kMaxHeads = 128;    // heads per launch (parameters travel by value)
+constexpr int kMaxTp = 256;       // limits of the in-kernel key-block bitmasks
+constexpr int kMaxSp = 2048;
+
+// Problem geometry handed to every kernel by value.
+struct Geom {
+  int T, H, W;             // real token grid
+  int bt, bh, bw;          // mask block (PSABlock) extents in tokens
+  int Tp, Hp, Wp, Sp, NB;  // block grid after 3D-padding; Sp = Hp*Wp, NB = Tp*Sp
+  int ct, ch, cw;          // 128-token slab = one TMA box (ct*ch*cw == 128)
+  int n_sub;               // slabs per mask block (1..3)
+  int sub_axis;            // axis along which the slabs of a block stack: 0 = t, 1 = h, 2 = w
+  int n_heads;
+  int items_per_block;     // work items per query block = ceil(n_sub / 2)
+  float scale_log2;        // softmax scale times log2(e)
+  long long L;             // T*H*W
+};
+
+struct HeadParamsArray {
+  psa_head_params p[kMaxHeads];
+};
+
+// One unit of work of the attention kernel: up to two query slabs of one query block.
+// x = head, y = query block id, z = number of attended key blocks,
+// w = first slab index | (number of slabs << 16)
+typedef int4 WorkItem;
+
+// Layout of the per-device workspace (all int32 words).
+constexpr int kWsStatus = 0;     // first device-side error (0 = none)
+constexpr int kWsDetail = 1;     // diagnostic of that error
+constexpr int kWsCounter = 2;    // dynamic scheduler ticket
+constexpr int kWsHeaderWords = 16;
+
+// One axis condition of the stripe mask (Algorithm 1): delta is key minus query
+// coordinate in blocks; stride 0 encodes an infinite stride.
+__host__ __device__ __forceinline__ bool axis_attends(int delta, int width, int offset, int stride) {
+  int x = delta - offset;
+  x = x < 0 ? -x : x;
+  if (stride != 0) x = x % stride;
+  return x <= width - 1;
+}
+
+}  // namespace psa

@@ -1,0 +1,353 @@
+// Host side of the PSA library: argument validation, geometry, per-device workspace,
+// TMA descriptors and the extern "C" entry points declared in psa.h.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <cmath>
+#include <cstring>
+#include <mutex>
+
+#include "psa_common.cuh"
+
+namespace psa {
+cudaError_t launch_mask_build(const HeadParamsArray& hp, const Geom& g, int head0, int n_heads_here,
+                              uint8_t* block_mask, int* row_ptr, int* col_idx, int ptr_base,
+                              int n_sms, cudaStream_t stream, int* launches);
+cudaError_t launch_plan(const HeadParamsArray& hp, const Geom& g, int head0, int n_heads_here, int* ws_header,
+                        psa_head_params* hp_dev, WorkItem* items, cudaStream_t stream);
+cudaError_t launch_attn(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to,
+                        const Geom& g, const WorkItem* items, const psa_head_params* hp_dev, int* ws_header,
+                        float* lse, int n_items, int n_sms, cudaStream_t stream);
+}  // namespace psa
+
+namespace {
+
+using namespace psa;
+
+std::atomic<long long> g_launches{0};
+std::mutex g_mu;
+
+constexpr int kMaxDevices = 64;
+struct Workspace {
+  void* base = nullptr;
+  size_t bytes = 0;
+  int n_sms = 0;
+  int cc_major = 0;
+};
+Workspace g_ws[kMaxDevices];
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode = nullptr;
+
+int load_driver_entry() {
+  if (g_encode) return PSA_OK;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+      qres != cudaDriverEntryPointSuccess || fn == nullptr) {
+    return PSA_ERR_CUDA;
+  }
+  g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+  return PSA_OK;
+}
+
+bool valid_params(const psa_head_params& p) {
+  const int lim = 1 << 30;
+  return p.Tw >= 1 && p.Sw >= 1 && p.Ts >= 0 && p.Ss >= 0 && p.To > -lim && p.To < lim && p.So > -lim && p.So < lim;
+}
+
+// Geometry of the block grid; `for_attn` additionally derives the 128-token slab.
+int make_geom(const psa_problem* prob, int T, int H, int W, bool for_attn, Geom* g) {
+  if (!prob || T < 1 || H < 1 || W < 1 || prob->n_heads < 1) return PSA_ERR_INVALID_ARG;
+  const psa_tile t = prob->tile;
+  if (t.bt < 1 || t.bh < 1 || t.bw < 1) return PSA_ERR_INVALID_ARG;
+  const long long L = (long long)T * H * W;
+  if (L >= (1ll << 31)) return PSA_ERR_INVALID_ARG;
+  std::memset(g, 0, sizeof(*g));
+  g->T = T; g->H = H; g->W = W;
+  g->bt = t.bt; g->bh = t.bh; g->bw = t.bw;
+  g->Tp = (T + t.bt - 1) / t.bt;
+  g->Hp = (H + t.bh - 1) / t.bh;
+  g->Wp = (W + t.bw - 1) / t.bw;
+  g->Sp = g->Hp * g->Wp;
+  const long long nb = (long long)g->Tp * g->Sp;
+  if (nb > (1 << 20)) return PSA_ERR_UNSUPPORTED;
+  g->NB = (int)nb;
+  g->n_heads = prob->n_heads;
+  g->L = L;
+  g->ct = t.bt; g->ch = t.bh; g->cw = t.bw;
+  g->n_sub = 1;
+  g->sub_axis = 0;
+  g->items_per_block = 1;
+  if (for_attn) {
+    if (prob->head_dim != kHeadDim) return PSA_ERR_UNSUPPORTED;
+    if (!(prob->scale > 0.f) || !std::isfinite(prob->scale)) return PSA_ERR_INVALID_ARG;
+    const long long tokens = (long long)t.bt * t.bh * t.bw;
+    if (tokens != 128 && tokens != 256 && tokens != 384) return PSA_ERR_UNSUPPORTED;
+    const int n_sub = (int)(tokens / kSlabTokens);
+    // split the block into n_sub slabs along its outermost axis of extent > 1
+    if (t.bt > 1 || (t.bh == 1 && t.bw == 1)) {
+      if (t.bt % n_sub) return PSA_ERR_UNSUPPORTED;
+      g->ct = t.bt / n_sub; g->sub_axis = 0;
+    } else if (t.bh > 1) {
+      if (t.bh % n_sub) return PSA_ERR_UNSUPPORTED;
+      g->ch = t.bh / n_sub; g->sub_axis = 1;
+    } else {
+      if (t.bw % n_sub) return PSA_ERR_UNSUPPORTED;
+      g->cw = t.bw / n_sub; g->sub_axis = 2;
+    }
+    if (g->ct > 128 || g->ch > 128 || g->cw > 128) return PSA_ERR_UNSUPPORTED;
+    if (g->Tp > kMaxTp || g->Sp > kMaxSp) return PSA_ERR_UNSUPPORTED;
+    g->n_sub = n_sub;
+    g->items_per_block = (n_sub + 1) / 2;
+    g->scale_log2 = prob->scale * 1.4426950408889634f;
+  }
+  return PSA_OK;
+}
+
+// Attended block pairs of one head: product of the two axis pair counts.
+long long head_nnz(const psa_head_params& p, const Geom& g) {
+  long long ct = 0, cs = 0;
+  for (int d = -(g.Tp - 1); d <= g.Tp - 1; ++d)
+    if (axis_attends(d, p.Tw, p.To, p.Ts)) ct += g.Tp - (d < 0 ? -d : d);
+  for (int d = -(g.Sp - 1); d <= g.Sp - 1; ++d)
+    if (axis_attends(d, p.Sw, p.So, p.Ss)) cs += g.Sp - (d < 0 ? -d : d);
+  return ct * cs;
+}
+
+int device_info(int* dev, Workspace** ws) {
+  if (cudaGetDevice(dev) != cudaSuccess) return PSA_ERR_CUDA;
+  if (*dev < 0 || *dev >= kMaxDevices) return PSA_ERR_UNSUPPORTED;
+  Workspace& w = g_ws[*dev];
+  if (w.n_sms == 0) {
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, *dev) != cudaSuccess) return PSA_ERR_CUDA;
+    w.n_sms = prop.multiProcessorCount;
+    w.cc_major = prop.major;
+  }
+  *ws = &w;
+  return PSA_OK;
+}
+
+int ensure_workspace(Workspace* w, size_t bytes) {
+  if (w->bytes >= bytes) return PSA_OK;
+  if (w->base) {
+    if (cudaDeviceSynchronize() != cudaSuccess) return PSA_ERR_CUDA;
+    cudaFree(w->base);
+    w->base = nullptr;
+    w->bytes = 0;
+  }
+  const size_t want = bytes + bytes / 4 + 4096;
+  if (cudaMalloc(&w->base, want) != cudaSuccess) return PSA_ERR_CUDA;
+  if (cudaMemset(w->base, 0, want) != cudaSuccess) return PSA_ERR_CUDA;
+  w->bytes = want;
+  return PSA_OK;
+}
+
+int encode_map(CUtensorMap* tm, const void* base, const Geom& g, const psa_problem* prob, int n_heads_here) {
+  const cuuint64_t dims[5] = {(cuuint64_t)kHeadDim, (cuuint64_t)g.W, (cuuint64_t)g.H, (cuuint64_t)g.T,
+                              (cuuint64_t)n_heads_here};
+  const cuuint64_t st = (cuuint64_t)prob->stride_token * 2;
+  const cuuint64_t strides[4] = {st, st * g.W, st * g.W * g.H,
+                                 n_heads_here > 1 ? (cuuint64_t)prob->stride_head * 2 : st * g.W * g.H * g.T};
+  const cuuint32_t box[5] = {64, (cuuint32_t)g.cw, (cuuint32_t)g.ch, (cuuint32_t)g.ct, 1};
+  const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+  const CUresult r = g_encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(base), dims, strides, box,
+                              estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? PSA_OK : PSA_ERR_INVALID_ARG;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+}  // namespace
+
+extern "C" {
+
+const char* psa_status_string(int status) {
+  switch (status) {
+    case PSA_OK: return "ok";
+    case PSA_ERR_INVALID_ARG: return "invalid argument";
+    case PSA_ERR_UNSUPPORTED: return "unsupported configuration";
+    case PSA_ERR_CAPACITY: return "col_idx capacity too small";
+    case PSA_ERR_CUDA: return "CUDA call failed";
+    case PSA_ERR_TIMEOUT: return "device-side wait timed out";
+    default: return "unknown status";
+  }
+}
+
+int64_t psa_launch_count(void) { return g_launches.load(); }
+
+int psa_mask_sizes(const psa_head_params* params, const psa_problem* prob, int T, int H, int W, int64_t* nb,
+                   int64_t* nnz) {
+  Geom g;
+  const int rc = make_geom(prob, T, H, W, false, &g);
+  if (rc != PSA_OK) return rc;
+  if (nb) *nb = g.NB;
+  if (nnz) {
+    if (!params) return PSA_ERR_INVALID_ARG;
+    long long tot = 0;
+    for (int h = 0; h < prob->n_heads; ++h) {
+      if (!valid_params(params[h])) return PSA_ERR_INVALID_ARG;
+      tot += head_nnz(params[h], g);
+    }
+    *nnz = tot;
+  }
+  return PSA_OK;
+}
+
+int psa_mask_build(const psa_head_params* params, const psa_problem* prob, int T, int H, int W, uint8_t* block_mask,
+                   int32_t* row_ptr, int32_t* col_idx, int64_t col_capacity, void* stream) {
+  Geom g;
+  int rc = make_geom(prob, T, H, W, false, &g);
+  if (rc != PSA_OK) return rc;
+  if (!params) return PSA_ERR_INVALID_ARG;
+  if (col_idx && !row_ptr) return PSA_ERR_INVALID_ARG;
+  if (block_mask && !aligned16(block_mask)) return PSA_ERR_INVALID_ARG;
+  if ((row_ptr && (reinterpret_cast<uintptr_t>(row_ptr) & 3u)) || (col_idx && (reinterpret_cast<uintptr_t>(col_idx) & 3u)))
+    return PSA_ERR_INVALID_ARG;
+  long long nnz = 0;
+  for (int h = 0; h < prob->n_heads; ++h) {
+    if (!valid_params(params[h])) return PSA_ERR_INVALID_ARG;
+    nnz += head_nnz(params[h], g);
+  }
+  if (nnz >= (1ll << 31) || (long long)prob->n_heads * g.NB >= (1ll << 31) - 1) return PSA_ERR_UNSUPPORTED;
+  if (col_idx && col_capacity < nnz) return PSA_ERR_CAPACITY;
+  int dev;
+  Workspace* ws;
+  std::lock_guard<std::mutex> lock(g_mu);
+  rc = device_info(&dev, &ws);
+  if (rc != PSA_OK) return rc;
+  long long ptr_base = 0;
+  for (int head0 = 0; head0 < prob->n_heads; head0 += kMaxHeads) {
+    const int n_here = prob->n_heads - head0 < kMaxHeads ? prob->n_heads - head0 : kMaxHeads;
+    HeadParamsArray hp;
+    std::memset(&hp, 0, sizeof(hp));
+    // kernels index hp.p[head0 + h] relative to the chunk: store the chunk at its own offset
+    for (int h = 0; h < n_here; ++h) hp.p[h] = params[head0 + h];
+    int launches = 0;
+    const cudaError_t e = launch_mask_build(hp, g, 0, n_here, block_mask ? block_mask + (long long)head0 * g.NB * g.NB : nullptr,
+                                            row_ptr ? row_ptr + (long long)head0 * g.NB : nullptr, col_idx, (int)ptr_base,
+                                            ws->n_sms, static_cast<cudaStream_t>(stream), &launches);
+    g_launches += launches;
+    if (e != cudaSuccess) return PSA_ERR_CUDA;
+    for (int h = 0; h < n_here; ++h) ptr_base += head_nnz(params[head0 + h], g);
+  }
+  return PSA_OK;
+}
+
+int psa_attn_fwd(const void* q, const void* k, const void* v, void* out, float* lse, const psa_head_params* head_params,
+                 const psa_problem* prob, int T, int H, int W, void* stream) {
+  Geom g;
+  int rc = make_geom(prob, T, H, W, true, &g);
+  if (rc != PSA_OK) return rc;
+  if (!q || !k || !v || !out || !lse || !head_params) return PSA_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || (reinterpret_cast<uintptr_t>(lse) & 3u))
+    return PSA_ERR_INVALID_ARG;
+  if (out == q || out == k || out == v) return PSA_ERR_INVALID_ARG;
+  if (prob->stride_token < kHeadDim || (prob->stride_token % 8) != 0) return PSA_ERR_INVALID_ARG;
+  if (prob->n_heads > 1 && (prob->stride_head < kHeadDim || (prob->stride_head % 8) != 0)) return PSA_ERR_INVALID_ARG;
+  for (int h = 0; h < prob->n_heads; ++h)
+    if (!valid_params(head_params[h])) return PSA_ERR_INVALID_ARG;
+
+  std::lock_guard<std::mutex> lock(g_mu);
+  int dev;
+  Workspace* ws;
+  rc = device_info(&dev, &ws);
+  if (rc != PSA_OK) return rc;
+  if (ws->cc_major != 10) return PSA_ERR_UNSUPPORTED;
+  rc = load_driver_entry();
+  if (rc != PSA_OK) return rc;
+
+  const int chunk = prob->n_heads < kMaxHeads ? prob->n_heads : kMaxHeads;
+  const size_t items_bytes = sizeof(WorkItem) * (size_t)chunk * g.NB * g.items_per_block;
+  const size_t hp_off = sizeof(int) * kWsHeaderWords;
+  const size_t items_off = (hp_off + sizeof(psa_head_params) * kMaxHeads + 255) & ~size_t(255);
+  rc = ensure_workspace(ws, items_off + items_bytes);
+  if (rc != PSA_OK) return rc;
+  int* ws_header = static_cast<int*>(ws->base);
+  psa_head_params* hp_dev = reinterpret_cast<psa_head_params*>(static_cast<char*>(ws->base) + hp_off);
+  WorkItem* items = reinterpret_cast<WorkItem*>(static_cast<char*>(ws->base) + items_off);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+
+  for (int head0 = 0; head0 < prob->n_heads; head0 += kMaxHeads) {
+    const int n_here = prob->n_heads - head0 < kMaxHeads ? prob->n_heads - head0 : kMaxHeads;
+    HeadParamsArray hp;
+    std::memset(&hp, 0, sizeof(hp));
+    for (int h = 0; h < n_here; ++h) hp.p[h] = head_params[head0 + h];
+    const long long eoff = (long long)head0 * prob->stride_head;
+    CUtensorMap tq, tk, tv, to;
+    if ((rc = encode_map(&tq, static_cast<const uint16_t*>(q) + eoff, g, prob, n_here)) != PSA_OK) return rc;
+    if ((rc = encode_map(&tk, static_cast<const uint16_t*>(k) + eoff, g, prob, n_here)) != PSA_OK) return rc;
+    if ((rc = encode_map(&tv, static_cast<const uint16_t*>(v) + eoff, g, prob, n_here)) != PSA_OK) return rc;
+    if ((rc = encode_map(&to, static_cast<uint16_t*>(out) + eoff, g, prob, n_here)) != PSA_OK) return rc;
+    Geom gh = g;
+    gh.n_heads = n_here;
+    if (launch_plan(hp, gh, 0, n_here, ws_header, hp_dev, items, st) != cudaSuccess) return PSA_ERR_CUDA;
+    ++g_launches;
+    const int n_items = n_here * g.NB * g.items_per_block;
+    if (launch_attn(tq, tk, tv, to, gh, items, hp_dev, ws_header, lse + (long long)head0 * g.L, n_items, ws->n_sms, st) !=
+        cudaSuccess)
+      return PSA_ERR_CUDA;
+    ++g_launches;
+  }
+  return PSA_OK;
+}
+
+int psa_attn_fwd_host(const void* q, const void* k, const void* v, void* out, float* lse, void* d_q, void* d_k, void* d_v,
+                      void* d_out, float* d_lse, const psa_head_params* head_params, const psa_problem* prob, int T, int H,
+                      int W, void* stream) {
+  if (!prob || !q || !k || !v || !out || !lse || !d_q || !d_k || !d_v || !d_out || !d_lse) return PSA_ERR_INVALID_ARG;
+  if (T < 1 || H < 1 || W < 1 || prob->n_heads < 1) return PSA_ERR_INVALID_ARG;
+  const long long L = (long long)T * H * W;
+  const size_t elems = (size_t)(prob->n_heads - 1) * prob->stride_head + (size_t)(L - 1) * prob->stride_token + prob->head_dim;
+  const size_t bytes = elems * 2;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (cudaMemcpyAsync(d_q, q, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return PSA_ERR_CUDA;
+  if (cudaMemcpyAsync(d_k, k, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return PSA_ERR_CUDA;
+  if (cudaMemcpyAsync(d_v, v, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return PSA_ERR_CUDA;
+  const int rc = psa_attn_fwd(d_q, d_k, d_v, d_out, d_lse, head_params, prob, T, H, W, stream);
+  if (rc != PSA_OK) return rc;
+  if (cudaMemcpyAsync(out, d_out, bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return PSA_ERR_CUDA;
+  if (cudaMemcpyAsync(lse, d_lse, sizeof(float) * (size_t)prob->n_heads * L, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+    return PSA_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return PSA_ERR_CUDA;
+  return PSA_OK;
+}
+
+int psa_last_device_status(int32_t* detail) {
+  std::lock_guard<std::mutex> lock(g_mu);
+  int dev;
+  Workspace* ws;
+  int rc = device_info(&dev, &ws);
+  if (rc != PSA_OK) return rc;
+  if (cudaDeviceSynchronize() != cudaSuccess) return PSA_ERR_CUDA;
+  if (detail) *detail = 0;
+  if (!ws->base) return PSA_OK;
+  int hdr[2] = {0, 0};
+  if (cudaMemcpy(hdr, ws->base, sizeof(hdr), cudaMemcpyDeviceToHost) != cudaSuccess) return PSA_ERR_CUDA;
+  if (detail) *detail = hdr[1];
+  return hdr[0];
+}
+
+int psa_shutdown(void) {
+  std::lock_guard<std::mutex> lock(g_mu);
+  int cur = 0;
+  if (cudaGetDevice(&cur) != cudaSuccess) return PSA_OK;  // no usable device: nothing was allocated
+  for (int d = 0; d < kMaxDevices; ++d) {
+    if (g_ws[d].base) {
+      cudaSetDevice(d);
+      cudaDeviceSynchronize();
+      cudaFree(g_ws[d].base);
+      g_ws[d].base = nullptr;
+      g_ws[d].bytes = 0;
+    }
+  }
+  cudaSetDevice(cur);
+  return PSA_OK;
+}
+
+}  // extern "C"
