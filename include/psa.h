@@ -109,6 +109,11 @@ int psa_attn_fwd_host(const void* q, const void* k, const void* v, void* out, fl
  * diagnostic code naming the wait that gave up. */
 int psa_last_device_status(int32_t* detail);
 
+/* Measurement hook: when both are non-NULL cudaEvent_t handles, every later psa_attn_fwd
+ * records `start` on its stream just before the attention kernel and `stop` just after
+ * it (the planning kernel stays outside the pair).  Pass NULL, NULL to switch it off. */
+int psa_profile_events(void* start_event, void* stop_event);
+
 /* Number of kernels the library has launched since load (all entry points). */
 int64_t psa_launch_count(void);
 

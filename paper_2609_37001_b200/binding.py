@@ -64,6 +64,8 @@ def lib() -> ctypes.CDLL:
         L.psa_attn_fwd_host.argtypes = [vp] * 10 + [hp, pp, i32, i32, i32, vp]
         L.psa_last_device_status.argtypes = [ctypes.POINTER(ctypes.c_int32)]
         L.psa_shutdown.argtypes = []
+        L.psa_profile_events.argtypes = [vp, vp]
+        L.psa_profile_events.restype = ctypes.c_int
         for f in (L.psa_mask_sizes, L.psa_mask_build, L.psa_attn_fwd, L.psa_attn_fwd_host,
                   L.psa_last_device_status, L.psa_shutdown):
             f.restype = ctypes.c_int
@@ -190,6 +192,14 @@ def psa_last_device_status() -> Tuple[int, int]:
     detail = ctypes.c_int32(0)
     st = lib().psa_last_device_status(ctypes.byref(detail))
     return st, detail.value
+
+
+def psa_profile_events(start: Optional[torch.cuda.Event], stop: Optional[torch.cuda.Event]) -> None:
+    """Record ``start``/``stop`` around the attention kernel of every later psa_attn_fwd (None, None: off).
+    The events must have been created with enable_timing=True and recorded once (so that they exist)."""
+    a = None if start is None else ctypes.c_void_p(start.cuda_event)
+    b = None if stop is None else ctypes.c_void_p(stop.cuda_event)
+    _check(lib().psa_profile_events(a, b), "psa_profile_events")
 
 
 def psa_launch_count() -> int:

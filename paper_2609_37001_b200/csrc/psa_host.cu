@@ -41,6 +41,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 EncodeTiledFn g_encode = nullptr;
+cudaEvent_t g_ev_start = nullptr, g_ev_stop = nullptr;
 
 int load_driver_entry() {
   if (g_encode) return PSA_OK;
@@ -181,6 +182,14 @@ const char* psa_status_string(int status) {
 
 int64_t psa_launch_count(void) { return g_launches.load(); }
 
+int psa_profile_events(void* start_event, void* stop_event) {
+  std::lock_guard<std::mutex> lock(g_mu);
+  if ((start_event == nullptr) != (stop_event == nullptr)) return PSA_ERR_INVALID_ARG;
+  g_ev_start = static_cast<cudaEvent_t>(start_event);
+  g_ev_stop = static_cast<cudaEvent_t>(stop_event);
+  return PSA_OK;
+}
+
 int psa_mask_sizes(const psa_head_params* params, const psa_problem* prob, int T, int H, int W, int64_t* nb,
                    int64_t* nnz) {
   Geom g;
@@ -289,9 +298,11 @@ int psa_attn_fwd(const void* q, const void* k, const void* v, void* out, float* 
     if (launch_plan(hp, gh, 0, n_here, ws_header, hp_dev, items, st) != cudaSuccess) return PSA_ERR_CUDA;
     ++g_launches;
     const int n_items = n_here * g.NB * g.items_per_block;
+    if (g_ev_start && g_ev_stop) cudaEventRecord(g_ev_start, st);
     if (launch_attn(tq, tk, tv, to, gh, items, hp_dev, ws_header, lse + (long long)head0 * g.L, n_items, ws->n_sms, st) !=
         cudaSuccess)
       return PSA_ERR_CUDA;
+    if (g_ev_start && g_ev_stop) cudaEventRecord(g_ev_stop, st);
     ++g_launches;
   }
   return PSA_OK;
