@@ -6,11 +6,13 @@
 // which the load warp enumerates in ascending block id straight from the six stripe
 // parameters (Algorithm 1) -- no mask or index list is read from memory.
 //
-// Roles (320 threads):
+// Roles (384 threads = 3 warpgroups):
 //   warps 0-3  softmax / correction / epilogue of query slab 0  (TMEM lanes 0..127)
 //   warps 4-7  the same for query slab 1
 //   warp  8    TMA loads: Q slabs once per item, K and V slabs through a 5-slot ring
 //   warp  9    tcgen05.mma issue: S_i = Q_i K^T (SS form), O_i += P_i V (P read from TMEM)
+//   warps 10-11 idle; they only exist so that the third warpgroup can hand its registers
+//              to the softmax warpgroups (setmaxnreg)
 // TMEM (512 columns): S0 | S1 | O0 | O1, 128 fp32 columns each; the bf16 probabilities
 // P_i overwrite the first 64 columns of S_i.
 // Every wait is bounded; on expiry the CTA records a status word and unwinds.
@@ -21,7 +23,7 @@
 
 namespace psa {
 
-constexpr int kThreads = 320;
+constexpr int kThreads = 384;                       // 3 warpgroups; register budgets are re-split below
 constexpr int kNumSlots = 5;                       // K/V ring slots of one 128 x 128 bf16 slab
 constexpr uint32_t kSlabBytes = 128 * 128 * 2;     // 32 KB
 constexpr uint32_t kHalfBytes = kSlabBytes / 2;    // one 64-column swizzled half
@@ -131,8 +133,7 @@ __device__ __forceinline__ void tc_mma_ts(uint32_t d, uint32_t a, uint64_t bdesc
       "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
       ::"r"(d), "r"(a), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
 }
-__device__ __forceinline__ void tc_ld32(uint32_t addr, float* v) {
-  uint32_t* r = reinterpret_cast<uint32_t*>(v);
+__device__ __forceinline__ void tc_ld32(uint32_t addr, uint32_t* r) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
       "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
@@ -143,8 +144,7 @@ __device__ __forceinline__ void tc_ld32(uint32_t addr, float* v) {
         "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
       : "r"(addr) : "memory");
 }
-__device__ __forceinline__ void tc_st32(uint32_t addr, const float* v) {
-  const uint32_t* r = reinterpret_cast<const uint32_t*>(v);
+__device__ __forceinline__ void tc_st32(uint32_t addr, const uint32_t* r) {
   asm volatile(
       "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
       "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
@@ -298,11 +298,14 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
 
+  if (warp >= 8) {
+  // Third warpgroup: give registers away (the budget is re-split per warpgroup).
+  asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
   if (warp == 8) {
     // ======================================================================= load warp
     uint32_t tile_g = 0;       // ring tiles issued so far (K and V alternate)
     uint32_t kv_g = 0;         // key slabs issued so far
-    uint32_t it_q[2] = {0, 0}; // items in which query slab i was active
+    uint32_t it_q0 = 0, it_q1 = 0; // items in which query slab i was active
     bool ok = true;
     for (int idx = blockIdx.x; ok && idx < prm.n_items; idx += gridDim.x) {
       const WorkItem wi = prm.items[idx];
@@ -322,8 +325,11 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       }
       __syncwarp();
       // query slabs
-      for (int i = 0; i < nq; ++i) {
-        ok = mbar_wait_warp(bar(kBarQEmpty + i), (it_q[i] & 1u) ^ 1u, abort_flag, 0x100 + i);
+#pragma unroll
+      for (int i = 0; i < 2; ++i) {
+        if (i >= nq) break;
+        const uint32_t itq = i == 0 ? it_q0 : it_q1;
+        ok = mbar_wait_warp(bar(kBarQEmpty + i), (itq & 1u) ^ 1u, abort_flag, 0x100 + i);
         if (!ok) break;
         if (lane == 0) {
           int t0, h0, w0;
@@ -333,7 +339,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           tma_load_5d(dst, &tm_q, bar(kBarQFull + i), 0, w0, h0, t0, head);
           tma_load_5d(dst + kHalfBytes, &tm_q, bar(kBarQFull + i), 64, w0, h0, t0, head);
         }
-        ++it_q[i];
+        if (i == 0) ++it_q0; else ++it_q1;
       }
       if (!ok) break;
       // key / value slabs in ascending key-block id
@@ -403,10 +409,12 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           if (globaltimer_ns() - t0 > kTimeoutNs) break;
         }
       }
+#pragma unroll
       for (int i = 0; i < 2; ++i) {
-        if (it_q[i] == 0) continue;
+        const uint32_t itq = i == 0 ? it_q0 : it_q1;
+        if (itq == 0) continue;
         const unsigned long long t0 = globaltimer_ns();
-        while (!mbar_try_wait(bar(kBarQFull + i), (it_q[i] - 1) & 1u)) {
+        while (!mbar_try_wait(bar(kBarQFull + i), (itq - 1) & 1u)) {
           if (globaltimer_ns() - t0 > kTimeoutNs) break;
         }
       }
@@ -417,8 +425,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     constexpr uint32_t kIdescQK = instr_desc(false);
     constexpr uint32_t kIdescPV = instr_desc(true);
     uint32_t tile_g = 0;
-    uint32_t it_q[2] = {0, 0};
-    uint32_t cnt_s[2] = {0, 0};  // S_i tiles produced; P_i tiles consumed so far
+    uint32_t it_q0 = 0, it_q1 = 0;
+    uint32_t cnt_s0 = 0, cnt_s1 = 0;  // P_i tiles consumed so far
     bool ok = true;
 
     // S_i = Q_i K^T over head_dim = 128: 8 MMAs of K = 16; both operands K-major, SW128.
@@ -449,11 +457,14 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       const WorkItem wi = prm.items[idx];
       const int nq = wi.w >> 16;
       const int n_kv = wi.z * g.n_sub;
-      for (int i = 0; i < nq; ++i) {
-        ok = mbar_wait_warp(bar(kBarQFull + i), it_q[i] & 1u, abort_flag, 0x200 + i);
+#pragma unroll
+      for (int i = 0; i < 2; ++i) {
+        if (i >= nq) break;
+        const uint32_t itq = i == 0 ? it_q0 : it_q1;
+        ok = mbar_wait_warp(bar(kBarQFull + i), itq & 1u, abort_flag, 0x200 + i);
         if (!ok) break;
         // the epilogue of the previous item must have drained O_i before it is overwritten
-        ok = mbar_wait_warp(bar(kBarOEmpty + i), (it_q[i] & 1u) ^ 1u, abort_flag, 0x202 + i);
+        ok = mbar_wait_warp(bar(kBarOEmpty + i), (itq & 1u) ^ 1u, abort_flag, 0x202 + i);
         if (!ok) break;
       }
       if (!ok) break;
@@ -465,9 +476,12 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           if (!ok) break;
           tc_fence_after();
           if (lane == 0) {
-            for (int i = 0; i < nq; ++i) {
-              issue_qk(i, slot);
-              tc_commit(bar(kBarSFull + i));
+#pragma unroll
+            for (int i = 0; i < 2; ++i) {
+              if (i < nq) {
+                issue_qk(i, slot);
+                tc_commit(bar(kBarSFull + i));
+              }
             }
             tc_commit(bar(kBarSlotEmpty + slot));
           }
@@ -488,10 +502,13 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             if (!ok) break;
             ++tile_g;
           }
-          for (int i = 0; ok && i < nq; ++i) {
-            ok = mbar_wait_warp(bar(kBarPReady + i), cnt_s[i] & 1u, abort_flag, 0x220 + i);
+#pragma unroll
+          for (int i = 0; i < 2; ++i) {
+            if (!ok || i >= nq) break;
+            const uint32_t cs = i == 0 ? cnt_s0 : cnt_s1;
+            ok = mbar_wait_warp(bar(kBarPReady + i), cs & 1u, abort_flag, 0x220 + i);
             if (!ok) break;
-            ++cnt_s[i];
+            if (i == 0) ++cnt_s0; else ++cnt_s1;
             tc_fence_after();
             if (lane == 0) {
               issue_pv(i, vslot, j > 0);
@@ -510,13 +527,17 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         if (!ok) break;
       } else {
         if (lane == 0) {
-          for (int i = 0; i < nq; ++i) tc_commit(bar(kBarOFull + i));
+          tc_commit(bar(kBarOFull + 0));
+          if (nq > 1) tc_commit(bar(kBarOFull + 1));
         }
         __syncwarp();
       }
-      for (int i = 0; i < nq; ++i) ++it_q[i];
+      ++it_q0;
+      if (nq > 1) ++it_q1;
     }
+  }
   } else {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
     // ======================================================================= softmax warps
     const int qi = warp >> 2;                     // query slab handled by this warpgroup
     const int row = (warp & 3) * 32 + lane;       // row of the slab == TMEM lane
@@ -542,7 +563,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         if (!ok) break;
         ++cnt_s;
         tc_fence_after();
-        float s[128];
+        uint32_t s[128];  // raw scores of this row (fp32 bit patterns), kept in registers
         tc_ld32(tS + 0, s + 0);
         tc_ld32(tS + 32, s + 32);
         tc_ld32(tS + 64, s + 64);
@@ -553,16 +574,22 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           const uint32_t v0 = m[1], v1 = m[2], v2 = m[3], v3 = m[4];
 #pragma unroll
           for (int c = 0; c < 32; ++c) {
-            if (!((v0 >> c) & 1u)) s[c] = neg_inf;
-            if (!((v1 >> c) & 1u)) s[32 + c] = neg_inf;
-            if (!((v2 >> c) & 1u)) s[64 + c] = neg_inf;
-            if (!((v3 >> c) & 1u)) s[96 + c] = neg_inf;
+            if (!((v0 >> c) & 1u)) s[c] = 0xff800000u;
+            if (!((v1 >> c) & 1u)) s[32 + c] = 0xff800000u;
+            if (!((v2 >> c) & 1u)) s[64 + c] = 0xff800000u;
+            if (!((v3 >> c) & 1u)) s[96 + c] = 0xff800000u;
           }
         }
-        float mx = s[0];
+        float mx0 = __uint_as_float(s[0]), mx1 = __uint_as_float(s[1]);
+        float mx2 = __uint_as_float(s[2]), mx3 = __uint_as_float(s[3]);
 #pragma unroll
-        for (int c = 1; c < 128; ++c) mx = fmaxf(mx, s[c]);
-        const float ms = mx * g.scale_log2;
+        for (int c = 4; c < 128; c += 4) {
+          mx0 = fmaxf(mx0, __uint_as_float(s[c]));
+          mx1 = fmaxf(mx1, __uint_as_float(s[c + 1]));
+          mx2 = fmaxf(mx2, __uint_as_float(s[c + 2]));
+          mx3 = fmaxf(mx3, __uint_as_float(s[c + 3]));
+        }
+        const float ms = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * g.scale_log2;
         // Lazy rescale: the reference maximum only moves when the new maximum exceeds
         // it by more than the threshold, so exponentials stay below 2^threshold.
         float alpha = 1.f;
@@ -575,28 +602,30 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           l *= alpha;
 #pragma unroll
           for (int c4 = 0; c4 < 4; ++c4) {
-            float o[32];
+            uint32_t o[32];
             tc_ld32(tO + c4 * 32, o);
             tc_wait_ld();
 #pragma unroll
-            for (int c = 0; c < 32; ++c) o[c] *= alpha;
+            for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
             tc_st32(tO + c4 * 32, o);
           }
         }
         const float m_use = (m_ref == neg_inf) ? 0.f : m_ref;
-        float sum = 0.f;
+        float sum0 = 0.f, sum1 = 0.f;
 #pragma unroll
         for (int c4 = 0; c4 < 4; ++c4) {
           uint32_t pk[16];
 #pragma unroll
           for (int c = 0; c < 16; ++c) {
-            const float p0 = fast_exp2(fmaf(s[c4 * 32 + 2 * c], g.scale_log2, -m_use));
-            const float p1 = fast_exp2(fmaf(s[c4 * 32 + 2 * c + 1], g.scale_log2, -m_use));
-            sum += p0 + p1;
+            const float p0 = fast_exp2(fmaf(__uint_as_float(s[c4 * 32 + 2 * c]), g.scale_log2, -m_use));
+            const float p1 = fast_exp2(fmaf(__uint_as_float(s[c4 * 32 + 2 * c + 1]), g.scale_log2, -m_use));
+            sum0 += p0;
+            sum1 += p1;
             pk[c] = pack_bf16(p0, p1);
           }
           tc_st16(tS + c4 * 16, pk);
         }
+        const float sum = sum0 + sum1;
         l += sum;
         tc_wait_st();
         tc_fence_before();
@@ -613,18 +642,21 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       uint8_t* stage = smem + kOffQ + (uint32_t)qi * kSlabBytes;
 #pragma unroll
       for (int c4 = 0; c4 < 4; ++c4) {
-        float o[32];
+        uint32_t o[32];
         if (n_kv > 0) {
           tc_ld32(tO + c4 * 32, o);
           tc_wait_ld();
+        } else {
+#pragma unroll
+          for (int c = 0; c < 32; ++c) o[c] = 0u;
         }
 #pragma unroll
         for (int c8 = 0; c8 < 4; ++c8) {
           uint32_t w[4];
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
-            const float a = empty ? 0.f : o[c8 * 8 + 2 * e] * inv;
-            const float b = empty ? 0.f : o[c8 * 8 + 2 * e + 1] * inv;
+            const float a = empty ? 0.f : __uint_as_float(o[c8 * 8 + 2 * e]) * inv;
+            const float b = empty ? 0.f : __uint_as_float(o[c8 * 8 + 2 * e + 1]) * inv;
             w[e] = pack_bf16(a, b);
           }
           // 128-byte swizzle of the staging slab: 16-byte chunk index xor (row mod 8)
