@@ -36,12 +36,14 @@ constexpr uint32_t kOffQ = 0;                                   // 2 slabs
 constexpr uint32_t kOffRing = 2 * kSlabBytes;                   // kNumSlots slabs
 constexpr uint32_t kOffBar = kOffRing + kNumSlots * kSlabBytes; // mbarriers
 constexpr int kBarQFull = 0, kBarQEmpty = 2, kBarSlotFull = 4, kBarSlotEmpty = 4 + kNumSlots,
-              kBarSFull = 4 + 2 * kNumSlots, kBarPReady = kBarSFull + 2, kBarOFull = kBarPReady + 2,
-              kBarOEmpty = kBarOFull + 2, kNumBars = kBarOEmpty + 2;
+              kBarSFull = 4 + 2 * kNumSlots, kBarPHalf = kBarSFull + 2, kBarPReady = kBarPHalf + 2,
+              kBarOFull = kBarPReady + 2, kBarOEmpty = kBarOFull + 2, kBarSchedFull = kBarOEmpty + 2,
+              kBarSchedEmpty = kBarSchedFull + 2, kNumBars = kBarSchedEmpty + 2;
 constexpr uint32_t kOffMeta = kOffBar + kNumBars * 8;           // kMetaRing x 8 words
 constexpr uint32_t kOffMaskT = kOffMeta + kMetaRing * 32;       // kMaxTp / 32 words
 constexpr uint32_t kOffMaskS = kOffMaskT + (kMaxTp / 32) * 4;   // kMaxSp / 32 words
-constexpr uint32_t kOffMisc = kOffMaskS + (kMaxSp / 32) * 4;    // tmem base, abort flag
+constexpr uint32_t kOffSched = kOffMaskS + (kMaxSp / 32) * 4;   // two published work items
+constexpr uint32_t kOffMisc = kOffSched + 32;                   // tmem base, abort flag
 constexpr uint32_t kSmemBytes = kOffMisc + 16;
 constexpr uint32_t kSmemAlloc = kSmemBytes + 1024;              // slack for manual alignment
 
@@ -121,6 +123,9 @@ __device__ __forceinline__ void tc_commit(uint32_t bar) {
 }
 // D[tmem] (+)= A[smem desc] * B[smem desc]
 __device__ __forceinline__ void tc_mma_ss(uint32_t d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+#ifdef PSA_DBG_NOMMA
+  return;
+#endif
   asm volatile(
       "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
@@ -128,6 +133,9 @@ __device__ __forceinline__ void tc_mma_ss(uint32_t d, uint64_t adesc, uint64_t b
 }
 // D[tmem] (+)= A[tmem] * B[smem desc]
 __device__ __forceinline__ void tc_mma_ts(uint32_t d, uint32_t a, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+#ifdef PSA_DBG_NOMMA
+  return;
+#endif
   asm volatile(
       "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
@@ -164,6 +172,9 @@ __device__ __forceinline__ void tc_st16(uint32_t addr, const uint32_t* r) {
       : "memory");
 }
 __device__ __forceinline__ float fast_exp2(float x) {
+#ifdef PSA_DBG_NOEXP
+  return x;
+#endif
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
@@ -187,8 +198,23 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
   return d;
 }
 // Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = 128; A is K-major.
+#ifdef PSA_DBG_N64
+constexpr uint32_t kDbgN = 64u;
+#else
+constexpr uint32_t kDbgN = 128u;
+#endif
 __host__ __device__ constexpr uint32_t instr_desc(bool b_mn_major) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((kDbgN >> 3) << 17) | ((128u >> 4) << 24);
+}
+// One elected lane of a converged warp (keeps the branch warp-uniform for the compiler).
+__device__ __forceinline__ bool elect_one() {
+#ifndef PSA_NO_ELECT
+  uint32_t pred;
+  asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(pred));
+  return pred != 0;
+#else
+  return (threadIdx.x & 31) == 0;
+#endif
 }
 
 // ----------------------------------------------------------------------------- planning
@@ -256,6 +282,14 @@ __device__ __forceinline__ void slab_origin(const Geom& g, int qb, int sub, int&
   else w0 += sub * g.cw;
 }
 
+// Descriptor halves.  Only the low word (start address, leading byte offset) changes
+// between MMAs; the high word (stride byte offset 1024, version, 128-byte swizzle) is fixed.
+constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
+__device__ __forceinline__ uint32_t desc_lo(uint32_t addr, uint32_t lbo_bytes) {
+  return ((addr >> 4) & 0x3FFFu) | ((lbo_bytes >> 4) << 16);
+}
+__device__ __forceinline__ uint64_t make_desc(uint32_t lo) { return ((uint64_t)kDescHi << 32) | lo; }
+
 __global__ void __launch_bounds__(kThreads, 1)
 attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                 const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o,
@@ -270,6 +304,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   uint32_t* meta = reinterpret_cast<uint32_t*>(smem + kOffMeta);
   uint32_t* maskT = reinterpret_cast<uint32_t*>(smem + kOffMaskT);
   uint32_t* maskS = reinterpret_cast<uint32_t*>(smem + kOffMaskS);
+  volatile int4* sched = reinterpret_cast<volatile int4*>(smem + kOffSched);
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + kOffMisc);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kOffMisc + 4);
 
@@ -279,9 +314,12 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       mbar_init(bar(kBarQFull + i), 1);
       mbar_init(bar(kBarQEmpty + i), 1);
       mbar_init(bar(kBarSFull + i), 1);
+      mbar_init(bar(kBarPHalf + i), 128);
       mbar_init(bar(kBarPReady + i), 128);
       mbar_init(bar(kBarOFull + i), 1);
       mbar_init(bar(kBarOEmpty + i), 128);
+      mbar_init(bar(kBarSchedFull + i), 1);
+      mbar_init(bar(kBarSchedEmpty + i), 9);  // the MMA warp and the eight softmax warps
     }
     for (int s = 0; s < kNumSlots; ++s) {
       mbar_init(bar(kBarSlotFull + s), 1);
@@ -296,7 +334,30 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  const uint32_t tmem = *tmem_slot;
+  // The CTA owns all 512 TMEM columns, so the allocation starts at column 0, lane 0; using
+  // the constant keeps every TMEM address of the MMA stream in uniform registers.  Checked:
+  // any other base is reported through the status word and the CTA does no work.
+  constexpr uint32_t tmem = 0u;
+  const bool tmem_ok = (*tmem_slot == 0u);
+  if (!tmem_ok && threadIdx.x == 0) atomicCAS((int*)abort_flag, 0, 0x500);
+
+  // Work items are handed out through a two-entry ring: the load warp draws a ticket from
+  // a global counter (items are stored heaviest first), publishes the item, and the other
+  // roles pick it up.  A negative head ends the kernel.
+  auto next_item = [&](uint32_t n, WorkItem& wi) -> bool {
+    const uint32_t slot = n & 1u;
+    if (!tmem_ok) return false;
+    if (!mbar_wait_warp(bar(kBarSchedFull + slot), (n >> 1) & 1u, abort_flag, 0x400)) return false;
+    // broadcast from lane 0 so that the compiler knows the item (and every loop bound
+    // derived from it) is warp-uniform
+    wi.x = __shfl_sync(0xffffffffu, sched[slot].x, 0);
+    wi.y = __shfl_sync(0xffffffffu, sched[slot].y, 0);
+    wi.z = __shfl_sync(0xffffffffu, sched[slot].z, 0);
+    wi.w = __shfl_sync(0xffffffffu, sched[slot].w, 0);
+    __syncwarp();
+    if (lane == 0) mbar_arrive(bar(kBarSchedEmpty + slot));
+    return wi.x >= 0;
+  };
 
   if (warp >= 8) {
   // Third warpgroup: give registers away (the budget is re-split per warpgroup).
@@ -306,9 +367,22 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     uint32_t tile_g = 0;       // ring tiles issued so far (K and V alternate)
     uint32_t kv_g = 0;         // key slabs issued so far
     uint32_t it_q0 = 0, it_q1 = 0; // items in which query slab i was active
-    bool ok = true;
-    for (int idx = blockIdx.x; ok && idx < prm.n_items; idx += gridDim.x) {
-      const WorkItem wi = prm.items[idx];
+    bool ok = tmem_ok;
+    for (uint32_t n = 0; ok; ++n) {
+      const uint32_t sslot = n & 1u;
+      ok = mbar_wait_warp(bar(kBarSchedEmpty + sslot), ((n >> 1) & 1u) ^ 1u, abort_flag, 0x401);
+      if (!ok) break;
+      WorkItem wi = make_int4(-1, 0, 0, 0);
+      if (lane == 0) {
+        const int ticket = atomicAdd(prm.ws_header + kWsCounter, 1);
+        if (ticket < prm.n_items) wi = prm.items[ticket];
+        sched[sslot].x = wi.x; sched[sslot].y = wi.y; sched[sslot].z = wi.z; sched[sslot].w = wi.w;
+        mbar_arrive(bar(kBarSchedFull + sslot));
+      }
+      wi.x = __shfl_sync(0xffffffffu, wi.x, 0);
+      wi.y = __shfl_sync(0xffffffffu, wi.y, 0);
+      wi.w = __shfl_sync(0xffffffffu, wi.w, 0);
+      if (wi.x < 0) break;
       const int head = wi.x, qb = wi.y, sub0 = wi.w & 0xffff, nq = wi.w >> 16;
       const psa_head_params p = prm.hp_dev[head];
       const int tq = qb / g.Sp, sq = qb % g.Sp;
@@ -359,14 +433,17 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 slab_origin(g, kb, sub, t0, h0, w0);
                 // validity of the slab's 128 key positions (3D-padding): bit c of word c/32
                 const bool edge = (t0 + g.ct > g.T) || (h0 + g.ch > g.H) || (w0 + g.cw > g.W);
-                uint32_t vw[4] = {0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu};
+                uint32_t vw0 = 0xffffffffu, vw1 = 0xffffffffu, vw2 = 0xffffffffu, vw3 = 0xffffffffu;
                 if (edge) {
-#pragma unroll
-                  for (int w4 = 0; w4 < 4; ++w4) {
-                    const int c = w4 * 32 + lane;
-                    const int wi_ = c % g.cw, hi_ = (c / g.cw) % g.ch, ti_ = c / (g.cw * g.ch);
-                    vw[w4] = __ballot_sync(0xffffffffu, (t0 + ti_ < g.T) && (h0 + hi_ < g.H) && (w0 + wi_ < g.W));
-                  }
+                  const int chw = g.cw * g.ch;
+                  int c = lane;
+                  vw0 = __ballot_sync(0xffffffffu, (t0 + c / chw < g.T) && (h0 + (c / g.cw) % g.ch < g.H) && (w0 + c % g.cw < g.W));
+                  c += 32;
+                  vw1 = __ballot_sync(0xffffffffu, (t0 + c / chw < g.T) && (h0 + (c / g.cw) % g.ch < g.H) && (w0 + c % g.cw < g.W));
+                  c += 32;
+                  vw2 = __ballot_sync(0xffffffffu, (t0 + c / chw < g.T) && (h0 + (c / g.cw) % g.ch < g.H) && (w0 + c % g.cw < g.W));
+                  c += 32;
+                  vw3 = __ballot_sync(0xffffffffu, (t0 + c / chw < g.T) && (h0 + (c / g.cw) % g.ch < g.H) && (w0 + c % g.cw < g.W));
                 }
                 const uint32_t sk_slot = tile_g % kNumSlots, sk_use = tile_g / kNumSlots;
                 ok = mbar_wait_warp(bar(kBarSlotEmpty + sk_slot), (sk_use & 1u) ^ 1u, abort_flag, 0x110);
@@ -374,11 +451,16 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 if (lane == 0) {
                   uint32_t* m = meta + (kv_g % kMetaRing) * 8;
                   m[0] = edge ? 1u : 0u;
-                  m[1] = vw[0]; m[2] = vw[1]; m[3] = vw[2]; m[4] = vw[3];
+                  m[1] = vw0; m[2] = vw1; m[3] = vw2; m[4] = vw3;
                   const uint32_t dst = sbase + kOffRing + sk_slot * kSlabBytes;
+#ifdef PSA_DBG_NOLOAD
+                  (void)dst;
+                  mbar_arrive(bar(kBarSlotFull + sk_slot));
+#else
                   mbar_expect_tx(bar(kBarSlotFull + sk_slot), kSlabBytes);
                   tma_load_5d(dst, &tm_k, bar(kBarSlotFull + sk_slot), 0, w0, h0, t0, head);
                   tma_load_5d(dst + kHalfBytes, &tm_k, bar(kBarSlotFull + sk_slot), 64, w0, h0, t0, head);
+#endif
                 }
                 ++tile_g;
                 const uint32_t sv_slot = tile_g % kNumSlots, sv_use = tile_g / kNumSlots;
@@ -386,9 +468,14 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 if (!ok) break;
                 if (lane == 0) {
                   const uint32_t dst = sbase + kOffRing + sv_slot * kSlabBytes;
+#ifdef PSA_DBG_NOLOAD
+                  (void)dst;
+                  mbar_arrive(bar(kBarSlotFull + sv_slot));
+#else
                   mbar_expect_tx(bar(kBarSlotFull + sv_slot), kSlabBytes);
                   tma_load_5d(dst, &tm_v, bar(kBarSlotFull + sv_slot), 0, w0, h0, t0, head);
                   tma_load_5d(dst + kHalfBytes, &tm_v, bar(kBarSlotFull + sv_slot), 64, w0, h0, t0, head);
+#endif
                 }
                 ++tile_g;
                 ++kv_g;
@@ -428,33 +515,43 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     uint32_t it_q0 = 0, it_q1 = 0;
     uint32_t cnt_s0 = 0, cnt_s1 = 0;  // P_i tiles consumed so far
     bool ok = true;
+    const uint32_t q_lo = desc_lo(sbase + kOffQ, 16);
+    const uint32_t ring_lo_k = desc_lo(sbase + kOffRing, 16);
+    const uint32_t ring_lo_v = desc_lo(sbase + kOffRing, kHalfBytes);
+    constexpr uint32_t kSlabStep = kSlabBytes >> 4;  // descriptor address units per slab
 
     // S_i = Q_i K^T over head_dim = 128: 8 MMAs of K = 16; both operands K-major, SW128.
     auto issue_qk = [&](int i, uint32_t kslot) {
-      const uint32_t qaddr = sbase + kOffQ + (uint32_t)i * kSlabBytes;
-      const uint32_t kaddr = sbase + kOffRing + kslot * kSlabBytes;
+#ifdef PSA_DBG_NOQK
+      return;
+#endif
+      const uint32_t a0 = q_lo + (uint32_t)i * kSlabStep, b0 = ring_lo_k + kslot * kSlabStep;
 #pragma unroll
       for (int kk = 0; kk < 8; ++kk) {
-        const uint32_t off = (uint32_t)(kk >> 2) * kHalfBytes + (uint32_t)(kk & 3) * 32u;
-        tc_mma_ss(tmem + (uint32_t)i * 128u, smem_desc(qaddr + off, 16, 1024), smem_desc(kaddr + off, 16, 1024),
-                  kIdescQK, kk > 0 ? 1u : 0u);
+        const uint32_t off = (uint32_t)(kk >> 2) * (kHalfBytes >> 4) + (uint32_t)(kk & 3) * 2u;
+        tc_mma_ss(tmem + (uint32_t)i * 128u, make_desc(a0 + off), make_desc(b0 + off), kIdescQK, kk > 0 ? 1u : 0u);
       }
     };
-    // O_i (+)= P_i V over 128 keys: 8 MMAs of K = 16; A = bf16 P in TMEM (8 columns per
-    // step), B = V slab as loaded (keys x head_dim, head_dim contiguous) = MN-major SW128:
-    // 16 keys advance 2048 bytes, the second 64 columns of head_dim sit one half further.
-    auto issue_pv = [&](int i, uint32_t vslot, bool accumulate) {
-      const uint32_t vaddr = sbase + kOffRing + vslot * kSlabBytes;
+    // O_i (+)= P_i V over keys [64*half, 64*half+64): 4 MMAs of K = 16; A = bf16 P in TMEM
+    // (8 columns per step), B = V slab as loaded (keys x head_dim, head_dim contiguous) =
+    // MN-major SW128: 16 keys advance 2048 bytes, the second 64 columns of head_dim sit one
+    // half slab further (leading byte offset).
+    auto issue_pv_half = [&](int i, uint32_t vslot, int half, bool accumulate) {
+#ifdef PSA_DBG_NOPV
+      return;
+#endif
+      const uint32_t b0 = ring_lo_v + vslot * kSlabStep;
 #pragma unroll
-      for (int kk = 0; kk < 8; ++kk) {
+      for (int k4 = 0; k4 < 4; ++k4) {
+        const int kk = half * 4 + k4;
         tc_mma_ts(tmem + 256u + (uint32_t)i * 128u, tmem + (uint32_t)i * 128u + (uint32_t)kk * 8u,
-                  smem_desc(vaddr + (uint32_t)kk * 2048u, kHalfBytes, 1024), kIdescPV,
-                  (accumulate || kk > 0) ? 1u : 0u);
+                  make_desc(b0 + (uint32_t)kk * (2048u >> 4)), kIdescPV, (accumulate || kk > 0) ? 1u : 0u);
       }
     };
 
-    for (int idx = blockIdx.x; ok && idx < prm.n_items; idx += gridDim.x) {
-      const WorkItem wi = prm.items[idx];
+    for (uint32_t n = 0; ok; ++n) {
+      WorkItem wi;
+      if (!next_item(n, wi)) break;
       const int nq = wi.w >> 16;
       const int n_kv = wi.z * g.n_sub;
 #pragma unroll
@@ -475,7 +572,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           ok = mbar_wait_warp(bar(kBarSlotFull + slot), use & 1u, abort_flag, 0x210);
           if (!ok) break;
           tc_fence_after();
-          if (lane == 0) {
+          if (elect_one()) {
 #pragma unroll
             for (int i = 0; i < 2; ++i) {
               if (i < nq) {
@@ -506,12 +603,20 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           for (int i = 0; i < 2; ++i) {
             if (!ok || i >= nq) break;
             const uint32_t cs = i == 0 ? cnt_s0 : cnt_s1;
-            ok = mbar_wait_warp(bar(kBarPReady + i), cs & 1u, abort_flag, 0x220 + i);
+#ifndef PSA_DBG_NOPWAIT
+            ok = mbar_wait_warp(bar(kBarPHalf + i), cs & 1u, abort_flag, 0x220 + i);
             if (!ok) break;
+#endif
+            tc_fence_after();
+            if (elect_one()) issue_pv_half(i, vslot, 0, j > 0);
+#ifndef PSA_DBG_NOPWAIT
+            ok = mbar_wait_warp(bar(kBarPReady + i), cs & 1u, abort_flag, 0x222 + i);
+            if (!ok) break;
+#endif
             if (i == 0) ++cnt_s0; else ++cnt_s1;
             tc_fence_after();
-            if (lane == 0) {
-              issue_pv(i, vslot, j > 0);
+            if (elect_one()) {
+              issue_pv_half(i, vslot, 1, true);
               if (i == nq - 1) tc_commit(bar(kBarSlotEmpty + vslot));
               if (more) {
                 issue_qk(i, kslot);
@@ -526,7 +631,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         }
         if (!ok) break;
       } else {
-        if (lane == 0) {
+        if (elect_one()) {
           tc_commit(bar(kBarOFull + 0));
           if (nq > 1) tc_commit(bar(kBarOFull + 1));
         }
@@ -548,8 +653,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     bool ok = true;
     const float neg_inf = __int_as_float(0xff800000);
 
-    for (int idx = blockIdx.x; ok && idx < prm.n_items; idx += gridDim.x) {
-      const WorkItem wi = prm.items[idx];
+    for (uint32_t n = 0; ok; ++n) {
+      WorkItem wi;
+      if (!next_item(n, wi)) break;
       const int head = wi.x, qb = wi.y, sub0 = wi.w & 0xffff, nq = wi.w >> 16;
       const int n_kv = wi.z * g.n_sub;
       if (qi >= nq) {
@@ -563,6 +669,12 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         if (!ok) break;
         ++cnt_s;
         tc_fence_after();
+#ifdef PSA_DBG_NOSOFTMAX
+        tc_fence_before();
+        mbar_arrive(bar(kBarPHalf + qi));
+        mbar_arrive(bar(kBarPReady + qi));
+        continue;
+#endif
         uint32_t s[128];  // raw scores of this row (fp32 bit patterns), kept in registers
         tc_ld32(tS + 0, s + 0);
         tc_ld32(tS + 32, s + 32);
@@ -612,24 +724,29 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         }
         const float m_use = (m_ref == neg_inf) ? 0.f : m_ref;
         float sum0 = 0.f, sum1 = 0.f;
+        // probabilities in two halves of 64 keys: the first P V MMAs start while the
+        // second half of the exponentials is still being computed
 #pragma unroll
-        for (int c4 = 0; c4 < 4; ++c4) {
-          uint32_t pk[16];
+        for (int half = 0; half < 2; ++half) {
 #pragma unroll
-          for (int c = 0; c < 16; ++c) {
-            const float p0 = fast_exp2(fmaf(__uint_as_float(s[c4 * 32 + 2 * c]), g.scale_log2, -m_use));
-            const float p1 = fast_exp2(fmaf(__uint_as_float(s[c4 * 32 + 2 * c + 1]), g.scale_log2, -m_use));
-            sum0 += p0;
-            sum1 += p1;
-            pk[c] = pack_bf16(p0, p1);
+          for (int c2 = 0; c2 < 2; ++c2) {
+            const int c4 = half * 2 + c2;
+            uint32_t pk[16];
+#pragma unroll
+            for (int c = 0; c < 16; ++c) {
+              const float p0 = fast_exp2(fmaf(__uint_as_float(s[c4 * 32 + 2 * c]), g.scale_log2, -m_use));
+              const float p1 = fast_exp2(fmaf(__uint_as_float(s[c4 * 32 + 2 * c + 1]), g.scale_log2, -m_use));
+              sum0 += p0;
+              sum1 += p1;
+              pk[c] = pack_bf16(p0, p1);
+            }
+            tc_st16(tS + c4 * 16, pk);
           }
-          tc_st16(tS + c4 * 16, pk);
+          tc_wait_st();
+          tc_fence_before();
+          mbar_arrive(bar((half == 0 ? kBarPHalf : kBarPReady) + qi));
         }
-        const float sum = sum0 + sum1;
-        l += sum;
-        tc_wait_st();
-        tc_fence_before();
-        mbar_arrive(bar(kBarPReady + qi));
+        l += sum0 + sum1;
       }
       if (!ok) break;
       // ---- epilogue: out = O / l, lse = ln2 * (m_ref + log2 l)
@@ -700,7 +817,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   }
   if (warp == 9) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(*tmem_slot), "r"(512) : "memory");
   }
 }
 
