@@ -35,10 +35,11 @@ constexpr unsigned long long kTimeoutNs = 2000000000ull;
 constexpr uint32_t kOffQ = 0;                                   // 2 slabs
 constexpr uint32_t kOffRing = 2 * kSlabBytes;                   // kNumSlots slabs
 constexpr uint32_t kOffBar = kOffRing + kNumSlots * kSlabBytes; // mbarriers
-constexpr int kBarQFull = 0, kBarQEmpty = 2, kBarSlotFull = 4, kBarSlotEmpty = 4 + kNumSlots,
-              kBarSFull = 4 + 2 * kNumSlots, kBarPHalf = kBarSFull + 2, kBarPReady = kBarPHalf + 2,
+constexpr int kNumPairBars = 3;
+constexpr int kBarQFull = 0, kBarQEmpty = 2, kBarPairFull = 4, kBarSlotEmpty = kBarPairFull + kNumPairBars,
+              kBarSFull = kBarSlotEmpty + kNumSlots, kBarPHalf = kBarSFull + 2, kBarPReady = kBarPHalf + 2,
               kBarOFull = kBarPReady + 2, kBarOEmpty = kBarOFull + 2, kBarSchedFull = kBarOEmpty + 2,
-              kBarSchedEmpty = kBarSchedFull + 2, kNumBars = kBarSchedEmpty + 2;
+              kBarSchedEmpty = kBarSchedFull + 2, kNumBars = (kBarSchedEmpty + 2 + 1) & ~1;
 constexpr uint32_t kOffMeta = kOffBar + kNumBars * 8;           // kMetaRing x 8 words
 constexpr uint32_t kOffMaskT = kOffMeta + kMetaRing * 32;       // kMaxTp / 32 words
 constexpr uint32_t kOffMaskS = kOffMaskT + (kMaxTp / 32) * 4;   // kMaxSp / 32 words
@@ -123,9 +124,6 @@ __device__ __forceinline__ void tc_commit(uint32_t bar) {
 }
 // D[tmem] (+)= A[smem desc] * B[smem desc]
 __device__ __forceinline__ void tc_mma_ss(uint32_t d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
-#ifdef PSA_DBG_NOMMA
-  return;
-#endif
   asm volatile(
       "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
@@ -133,9 +131,6 @@ __device__ __forceinline__ void tc_mma_ss(uint32_t d, uint64_t adesc, uint64_t b
 }
 // D[tmem] (+)= A[tmem] * B[smem desc]
 __device__ __forceinline__ void tc_mma_ts(uint32_t d, uint32_t a, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
-#ifdef PSA_DBG_NOMMA
-  return;
-#endif
   asm volatile(
       "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
@@ -172,13 +167,66 @@ __device__ __forceinline__ void tc_st16(uint32_t addr, const uint32_t* r) {
       : "memory");
 }
 __device__ __forceinline__ float fast_exp2(float x) {
-#ifdef PSA_DBG_NOEXP
-  return x;
-#endif
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+// packed fp32 pairs (one instruction for two lanes of work on sm_100)
+__device__ __forceinline__ uint64_t pack2(float a, float b) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+  return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& a, float& b) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t r;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+  return r;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float r;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
+}
+// 2^x for a pair on the FMA/ALU pipes: x = n + f with n = rint(x), f in [-0.5, 0.5];
+// 2^f by a cubic (relative error < 8e-5, far below the bf16 rounding of the result), and
+// 2^n by adding n to the exponent field.  x is clamped at -125 so the exponent cannot wrap.
+__device__ __forceinline__ void exp2_poly_pair(uint64_t x2, float& p0, float& p1) {
+  float x0, x1;
+  unpack2(x2, x0, x1);
+  x0 = fmaxf(x0, -125.f);
+  x1 = fmaxf(x1, -125.f);
+  const uint64_t xc = pack2(x0, x1);
+  const uint64_t magic = pack2(12582912.f, 12582912.f);       // 1.5 * 2^23: rounds to integer
+  const uint64_t t2 = add2(xc, magic);
+  const uint64_t n2 = add2(t2, pack2(-12582912.f, -12582912.f));
+  const uint64_t f2 = fma2(n2, pack2(-1.f, -1.f), xc);
+  uint64_t q2 = fma2(f2, pack2(0.05508868396282196f, 0.05508868396282196f), pack2(0.24260404706001282f, 0.24260404706001282f));
+  q2 = fma2(q2, f2, pack2(0.6932762265205383f, 0.6932762265205383f));
+  q2 = fma2(q2, f2, pack2(0.9999289512634277f, 0.9999289512634277f));
+  float q0, q1, t0, t1;
+  unpack2(q2, q0, q1);
+  unpack2(t2, t0, t1);
+  p0 = __int_as_float(__float_as_int(q0) + (__float_as_int(t0) << 23));
+  p1 = __int_as_float(__float_as_int(q1) + (__float_as_int(t1) << 23));
+}
+#ifndef PSA_EMU_PAIRS
+#define PSA_EMU_PAIRS 1   // of every 4 pairs of probabilities, this many use exp2_poly_pair
+#endif
+#ifndef PSA_SPLIT_P
+#define PSA_SPLIT_P 1     // publish P in two halves of 64 keys
+#endif
+#ifndef PSA_OPTIMISTIC
+#define PSA_OPTIMISTIC 0  // exponentiate with the running maximum before the slab maximum is known
+#endif
+
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
@@ -198,23 +246,14 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
   return d;
 }
 // Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = 128; A is K-major.
-#ifdef PSA_DBG_N64
-constexpr uint32_t kDbgN = 64u;
-#else
-constexpr uint32_t kDbgN = 128u;
-#endif
 __host__ __device__ constexpr uint32_t instr_desc(bool b_mn_major) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((kDbgN >> 3) << 17) | ((128u >> 4) << 24);
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
 }
 // One elected lane of a converged warp (keeps the branch warp-uniform for the compiler).
 __device__ __forceinline__ bool elect_one() {
-#ifndef PSA_NO_ELECT
   uint32_t pred;
   asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(pred));
   return pred != 0;
-#else
-  return (threadIdx.x & 31) == 0;
-#endif
 }
 
 // ----------------------------------------------------------------------------- planning
@@ -321,10 +360,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       mbar_init(bar(kBarSchedFull + i), 1);
       mbar_init(bar(kBarSchedEmpty + i), 9);  // the MMA warp and the eight softmax warps
     }
-    for (int s = 0; s < kNumSlots; ++s) {
-      mbar_init(bar(kBarSlotFull + s), 1);
-      mbar_init(bar(kBarSlotEmpty + s), 1);
-    }
+    for (int s = 0; s < kNumPairBars; ++s) mbar_init(bar(kBarPairFull + s), 1);
+    for (int s = 0; s < kNumSlots; ++s) mbar_init(bar(kBarSlotEmpty + s), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 9) {
@@ -364,7 +401,11 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
   if (warp == 8) {
     // ======================================================================= load warp
-    uint32_t tile_g = 0;       // ring tiles issued so far (K and V alternate)
+    // Ring tiles are issued in the order K_0, V_0, K_1, V_1, ...; the MMA warp needs V_j and
+    // K_{j+1} at the same moment, so those two travel under one "pair" barrier
+    // (K_0 and the last V of an item travel alone).
+    uint32_t tile_g = 0;       // ring tiles issued so far
+    uint32_t pair_g = 0;       // pair barriers armed so far
     uint32_t kv_g = 0;         // key slabs issued so far
     uint32_t it_q0 = 0, it_q1 = 0; // items in which query slab i was active
     bool ok = tmem_ok;
@@ -417,6 +458,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       }
       if (!ok) break;
       // key / value slabs in ascending key-block id
+      bool have_prev = false;
+      int pt0 = 0, ph0 = 0, pw0 = 0;  // origin of the previous slab (its V is still to be loaded)
       for (int tw = 0; ok && tw < g.Tp; tw += 32) {
         uint32_t mt = maskT[tw >> 5];
         while (ok && mt) {
@@ -445,54 +488,64 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                   c += 32;
                   vw3 = __ballot_sync(0xffffffffu, (t0 + c / chw < g.T) && (h0 + (c / g.cw) % g.ch < g.H) && (w0 + c % g.cw < g.W));
                 }
-                const uint32_t sk_slot = tile_g % kNumSlots, sk_use = tile_g / kNumSlots;
-                ok = mbar_wait_warp(bar(kBarSlotEmpty + sk_slot), (sk_use & 1u) ^ 1u, abort_flag, 0x110);
+                // slots: [V of the previous slab,] K of this slab
+                const uint32_t v_slot = tile_g % kNumSlots, v_use = tile_g / kNumSlots;
+                const uint32_t k_tile = tile_g + (have_prev ? 1u : 0u);
+                const uint32_t k_slot = k_tile % kNumSlots, k_use = k_tile / kNumSlots;
+                if (have_prev) {
+                  ok = mbar_wait_warp(bar(kBarSlotEmpty + v_slot), (v_use & 1u) ^ 1u, abort_flag, 0x111);
+                  if (!ok) break;
+                }
+                ok = mbar_wait_warp(bar(kBarSlotEmpty + k_slot), (k_use & 1u) ^ 1u, abort_flag, 0x110);
                 if (!ok) break;
                 if (lane == 0) {
                   uint32_t* m = meta + (kv_g % kMetaRing) * 8;
                   m[0] = edge ? 1u : 0u;
                   m[1] = vw0; m[2] = vw1; m[3] = vw2; m[4] = vw3;
-                  const uint32_t dst = sbase + kOffRing + sk_slot * kSlabBytes;
-#ifdef PSA_DBG_NOLOAD
-                  (void)dst;
-                  mbar_arrive(bar(kBarSlotFull + sk_slot));
-#else
-                  mbar_expect_tx(bar(kBarSlotFull + sk_slot), kSlabBytes);
-                  tma_load_5d(dst, &tm_k, bar(kBarSlotFull + sk_slot), 0, w0, h0, t0, head);
-                  tma_load_5d(dst + kHalfBytes, &tm_k, bar(kBarSlotFull + sk_slot), 64, w0, h0, t0, head);
-#endif
+                  const uint32_t pb = bar(kBarPairFull + pair_g % kNumPairBars);
+                  mbar_expect_tx(pb, have_prev ? 2u * kSlabBytes : kSlabBytes);
+                  if (have_prev) {
+                    const uint32_t dv = sbase + kOffRing + v_slot * kSlabBytes;
+                    tma_load_5d(dv, &tm_v, pb, 0, pw0, ph0, pt0, head);
+                    tma_load_5d(dv + kHalfBytes, &tm_v, pb, 64, pw0, ph0, pt0, head);
+                  }
+                  const uint32_t dk = sbase + kOffRing + k_slot * kSlabBytes;
+                  tma_load_5d(dk, &tm_k, pb, 0, w0, h0, t0, head);
+                  tma_load_5d(dk + kHalfBytes, &tm_k, pb, 64, w0, h0, t0, head);
                 }
-                ++tile_g;
-                const uint32_t sv_slot = tile_g % kNumSlots, sv_use = tile_g / kNumSlots;
-                ok = mbar_wait_warp(bar(kBarSlotEmpty + sv_slot), (sv_use & 1u) ^ 1u, abort_flag, 0x111);
-                if (!ok) break;
-                if (lane == 0) {
-                  const uint32_t dst = sbase + kOffRing + sv_slot * kSlabBytes;
-#ifdef PSA_DBG_NOLOAD
-                  (void)dst;
-                  mbar_arrive(bar(kBarSlotFull + sv_slot));
-#else
-                  mbar_expect_tx(bar(kBarSlotFull + sv_slot), kSlabBytes);
-                  tma_load_5d(dst, &tm_v, bar(kBarSlotFull + sv_slot), 0, w0, h0, t0, head);
-                  tma_load_5d(dst + kHalfBytes, &tm_v, bar(kBarSlotFull + sv_slot), 64, w0, h0, t0, head);
-#endif
-                }
-                ++tile_g;
+                tile_g = k_tile + 1;
+                ++pair_g;
                 ++kv_g;
+                have_prev = true;
+                pt0 = t0; ph0 = h0; pw0 = w0;
               }
             }
           }
         }
       }
+      if (ok && have_prev) {  // V of the item's last slab
+        const uint32_t v_slot = tile_g % kNumSlots, v_use = tile_g / kNumSlots;
+        ok = mbar_wait_warp(bar(kBarSlotEmpty + v_slot), (v_use & 1u) ^ 1u, abort_flag, 0x112);
+        if (!ok) break;
+        if (lane == 0) {
+          const uint32_t pb = bar(kBarPairFull + pair_g % kNumPairBars);
+          mbar_expect_tx(pb, kSlabBytes);
+          const uint32_t dv = sbase + kOffRing + v_slot * kSlabBytes;
+          tma_load_5d(dv, &tm_v, pb, 0, pw0, ph0, pt0, head);
+          tma_load_5d(dv + kHalfBytes, &tm_v, pb, 64, pw0, ph0, pt0, head);
+        }
+        ++tile_g;
+        ++pair_g;
+      }
     }
-    // Let every load that was issued land before the CTA retires: wait for each slot's
-    // last issued phase (bounded; the abort flag no longer cuts these short).
+    // Let every load that was issued land before the CTA retires: wait for the last armed
+    // phase of each pair barrier and of the Q barriers (bounded; the abort flag no longer
+    // cuts these short).
     if (lane == 0) {
-      for (uint32_t back = 0; back < (uint32_t)kNumSlots && back < tile_g; ++back) {
-        const uint32_t tg = tile_g - 1 - back;
-        const uint32_t slot = tg % kNumSlots, use = tg / kNumSlots;
+      for (uint32_t back = 0; back < (uint32_t)kNumPairBars && back < pair_g; ++back) {
+        const uint32_t pg = pair_g - 1 - back;
         const unsigned long long t0 = globaltimer_ns();
-        while (!mbar_try_wait(bar(kBarSlotFull + slot), use & 1u)) {
+        while (!mbar_try_wait(bar(kBarPairFull + pg % kNumPairBars), (pg / kNumPairBars) & 1u)) {
           if (globaltimer_ns() - t0 > kTimeoutNs) break;
         }
       }
@@ -511,7 +564,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     // ======================================================================= MMA warp
     constexpr uint32_t kIdescQK = instr_desc(false);
     constexpr uint32_t kIdescPV = instr_desc(true);
-    uint32_t tile_g = 0;
+    uint32_t tile_g = 0, pair_g = 0;
     uint32_t it_q0 = 0, it_q1 = 0;
     uint32_t cnt_s0 = 0, cnt_s1 = 0;  // P_i tiles consumed so far
     bool ok = true;
@@ -522,9 +575,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 
     // S_i = Q_i K^T over head_dim = 128: 8 MMAs of K = 16; both operands K-major, SW128.
     auto issue_qk = [&](int i, uint32_t kslot) {
-#ifdef PSA_DBG_NOQK
-      return;
-#endif
       const uint32_t a0 = q_lo + (uint32_t)i * kSlabStep, b0 = ring_lo_k + kslot * kSlabStep;
 #pragma unroll
       for (int kk = 0; kk < 8; ++kk) {
@@ -532,14 +582,11 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         tc_mma_ss(tmem + (uint32_t)i * 128u, make_desc(a0 + off), make_desc(b0 + off), kIdescQK, kk > 0 ? 1u : 0u);
       }
     };
-    // O_i (+)= P_i V over keys [64*half, 64*half+64): 4 MMAs of K = 16; A = bf16 P in TMEM
-    // (8 columns per step), B = V slab as loaded (keys x head_dim, head_dim contiguous) =
-    // MN-major SW128: 16 keys advance 2048 bytes, the second 64 columns of head_dim sit one
-    // half slab further (leading byte offset).
+    // O_i (+)= P_i V over 128 keys: 8 MMAs of K = 16; A = bf16 P in TMEM (8 columns per
+    // step), B = V slab as loaded (keys x head_dim, head_dim contiguous) = MN-major SW128:
+    // 16 keys advance 2048 bytes, the second 64 columns of head_dim sit one half slab
+    // further (leading byte offset).
     auto issue_pv_half = [&](int i, uint32_t vslot, int half, bool accumulate) {
-#ifdef PSA_DBG_NOPV
-      return;
-#endif
       const uint32_t b0 = ring_lo_v + vslot * kSlabStep;
 #pragma unroll
       for (int k4 = 0; k4 < 4; ++k4) {
@@ -568,9 +615,11 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       if (n_kv > 0) {
         // first key slab: both S tiles
         {
-          const uint32_t slot = tile_g % kNumSlots, use = tile_g / kNumSlots;
-          ok = mbar_wait_warp(bar(kBarSlotFull + slot), use & 1u, abort_flag, 0x210);
+          ok = mbar_wait_warp(bar(kBarPairFull + pair_g % kNumPairBars), (pair_g / kNumPairBars) & 1u, abort_flag, 0x210);
           if (!ok) break;
+          ++pair_g;
+          const uint32_t slot = tile_g % kNumSlots;
+          ++tile_g;
           tc_fence_after();
           if (elect_one()) {
 #pragma unroll
@@ -583,40 +632,37 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             tc_commit(bar(kBarSlotEmpty + slot));
           }
           __syncwarp();
-          ++tile_g;
         }
         for (int j = 0; ok && j < n_kv; ++j) {
-          const uint32_t vslot = tile_g % kNumSlots, vuse = tile_g / kNumSlots;
-          ok = mbar_wait_warp(bar(kBarSlotFull + vslot), vuse & 1u, abort_flag, 0x211);
+          // V_j and (unless this is the last slab) K_{j+1} arrive under one barrier
+          ok = mbar_wait_warp(bar(kBarPairFull + pair_g % kNumPairBars), (pair_g / kNumPairBars) & 1u, abort_flag, 0x211);
           if (!ok) break;
-          ++tile_g;
+          ++pair_g;
           const bool more = (j + 1 < n_kv);
-          uint32_t kslot = 0;
-          if (more) {
-            kslot = tile_g % kNumSlots;
-            const uint32_t kuse = tile_g / kNumSlots;
-            ok = mbar_wait_warp(bar(kBarSlotFull + kslot), kuse & 1u, abort_flag, 0x212);
-            if (!ok) break;
-            ++tile_g;
-          }
+          const uint32_t vslot = tile_g % kNumSlots;
+          const uint32_t kslot = (tile_g + 1) % kNumSlots;
+          tile_g += more ? 2u : 1u;
 #pragma unroll
           for (int i = 0; i < 2; ++i) {
             if (!ok || i >= nq) break;
             const uint32_t cs = i == 0 ? cnt_s0 : cnt_s1;
-#ifndef PSA_DBG_NOPWAIT
-            ok = mbar_wait_warp(bar(kBarPHalf + i), cs & 1u, abort_flag, 0x220 + i);
+#if PSA_SPLIT_P
+            ok = mbar_wait_warp(bar(kBarPHalf + i), cs & 1u, abort_flag, 0x224 + i);
             if (!ok) break;
-#endif
             tc_fence_after();
             if (elect_one()) issue_pv_half(i, vslot, 0, j > 0);
-#ifndef PSA_DBG_NOPWAIT
-            ok = mbar_wait_warp(bar(kBarPReady + i), cs & 1u, abort_flag, 0x222 + i);
-            if (!ok) break;
 #endif
+            ok = mbar_wait_warp(bar(kBarPReady + i), cs & 1u, abort_flag, 0x220 + i);
+            if (!ok) break;
             if (i == 0) ++cnt_s0; else ++cnt_s1;
             tc_fence_after();
             if (elect_one()) {
+#if PSA_SPLIT_P
               issue_pv_half(i, vslot, 1, true);
+#else
+              issue_pv_half(i, vslot, 0, j > 0);
+              issue_pv_half(i, vslot, 1, true);
+#endif
               if (i == nq - 1) tc_commit(bar(kBarSlotEmpty + vslot));
               if (more) {
                 issue_qk(i, kslot);
@@ -652,6 +698,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     uint32_t it_q = 0, cnt_s = 0, kv_g = 0;
     bool ok = true;
     const float neg_inf = __int_as_float(0xff800000);
+    const uint64_t sc2 = pack2(g.scale_log2, g.scale_log2);
 
     for (uint32_t n = 0; ok; ++n) {
       WorkItem wi;
@@ -669,12 +716,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         if (!ok) break;
         ++cnt_s;
         tc_fence_after();
-#ifdef PSA_DBG_NOSOFTMAX
-        tc_fence_before();
-        mbar_arrive(bar(kBarPHalf + qi));
-        mbar_arrive(bar(kBarPReady + qi));
-        continue;
-#endif
         uint32_t s[128];  // raw scores of this row (fp32 bit patterns), kept in registers
         tc_ld32(tS + 0, s + 0);
         tc_ld32(tS + 32, s + 32);
@@ -692,25 +733,93 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             if (!((v3 >> c) & 1u)) s[96 + c] = 0xff800000u;
           }
         }
-        float mx0 = __uint_as_float(s[0]), mx1 = __uint_as_float(s[1]);
-        float mx2 = __uint_as_float(s[2]), mx3 = __uint_as_float(s[3]);
+        // One pass over the row: probabilities exp2(scale*s - m_use) are written to TMEM as
+        // bf16 while the row maximum is gathered on the side.  Returns the row sum.
+        auto exp_pass = [&](float m_use, float& row_max, bool signal_half) -> float {
+          const uint64_t negm2 = pack2(-m_use, -m_use);
+          uint64_t sum2 = pack2(0.f, 0.f);
+          float mx0 = neg_inf, mx1 = neg_inf, mx2 = neg_inf, mx3 = neg_inf;
 #pragma unroll
-        for (int c = 4; c < 128; c += 4) {
-          mx0 = fmaxf(mx0, __uint_as_float(s[c]));
-          mx1 = fmaxf(mx1, __uint_as_float(s[c + 1]));
-          mx2 = fmaxf(mx2, __uint_as_float(s[c + 2]));
-          mx3 = fmaxf(mx3, __uint_as_float(s[c + 3]));
+          for (int c4 = 0; c4 < 4; ++c4) {
+            uint32_t pk[16];
+#pragma unroll
+            for (int c = 0; c < 16; ++c) {
+              const float s0 = __uint_as_float(s[c4 * 32 + 2 * c]), s1 = __uint_as_float(s[c4 * 32 + 2 * c + 1]);
+              if ((c & 3) == 0) mx0 = max3(mx0, s0, s1);
+              else if ((c & 3) == 1) mx1 = max3(mx1, s0, s1);
+              else if ((c & 3) == 2) mx2 = max3(mx2, s0, s1);
+              else mx3 = max3(mx3, s0, s1);
+              const uint64_t x2 = fma2(pack2(s0, s1), sc2, negm2);
+              float p0, p1;
+              if ((c & 3) < PSA_EMU_PAIRS) {
+                exp2_poly_pair(x2, p0, p1);
+              } else {
+                float x0, x1;
+                unpack2(x2, x0, x1);
+                p0 = fast_exp2(x0);
+                p1 = fast_exp2(x1);
+              }
+              sum2 = add2(sum2, pack2(p0, p1));
+              pk[c] = pack_bf16(p0, p1);
+            }
+            tc_st16(tS + c4 * 16, pk);
+#if PSA_SPLIT_P
+            if (c4 == 1 && signal_half) {  // first 64 keys are final: their P V MMAs may start
+              tc_wait_st();
+              tc_fence_before();
+              mbar_arrive(bar(kBarPHalf + qi));
+            }
+#endif
+          }
+          row_max = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+          float sum0, sum1;
+          unpack2(sum2, sum0, sum1);
+          return sum0 + sum1;
+        };
+        float sum, mx;
+        bool redo;
+        if (j == 0) {
+          // first slab of the item: the reference maximum is the row maximum itself
+          float a0 = neg_inf, a1 = neg_inf, a2 = neg_inf, a3 = neg_inf;
+#pragma unroll
+          for (int c = 0; c < 128; c += 8) {
+            a0 = max3(a0, __uint_as_float(s[c]), __uint_as_float(s[c + 1]));
+            a1 = max3(a1, __uint_as_float(s[c + 2]), __uint_as_float(s[c + 3]));
+            a2 = max3(a2, __uint_as_float(s[c + 4]), __uint_as_float(s[c + 5]));
+            a3 = max3(a3, __uint_as_float(s[c + 6]), __uint_as_float(s[c + 7]));
+          }
+          m_ref = fmaxf(fmaxf(a0, a1), fmaxf(a2, a3)) * g.scale_log2;
+          sum = exp_pass(m_ref == neg_inf ? 0.f : m_ref, mx, true);
+          redo = false;
+        } else {
+#if PSA_OPTIMISTIC
+          // Optimistic pass with the running reference maximum: exponentials start right
+          // after the load instead of after a full max reduction.  The reference only has to
+          // keep exp2 bounded; it moves (lazy rescale) when the slab's maximum exceeds it by
+          // more than the threshold, which is detected here and repaired below.
+          sum = exp_pass(m_ref == neg_inf ? 0.f : m_ref, mx, false);
+          redo = __any_sync(0xffffffffu, mx * g.scale_log2 > m_ref + kRescaleThreshold);
+#else
+          float a0 = neg_inf, a1 = neg_inf, a2 = neg_inf, a3 = neg_inf;
+#pragma unroll
+          for (int c = 0; c < 128; c += 8) {
+            a0 = max3(a0, __uint_as_float(s[c]), __uint_as_float(s[c + 1]));
+            a1 = max3(a1, __uint_as_float(s[c + 2]), __uint_as_float(s[c + 3]));
+            a2 = max3(a2, __uint_as_float(s[c + 4]), __uint_as_float(s[c + 5]));
+            a3 = max3(a3, __uint_as_float(s[c + 6]), __uint_as_float(s[c + 7]));
+          }
+          mx = fmaxf(fmaxf(a0, a1), fmaxf(a2, a3));
+          redo = __any_sync(0xffffffffu, mx * g.scale_log2 > m_ref + kRescaleThreshold);
+          if (!redo) sum = exp_pass(m_ref == neg_inf ? 0.f : m_ref, mx, true);
+#endif
         }
-        const float ms = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * g.scale_log2;
-        // Lazy rescale: the reference maximum only moves when the new maximum exceeds
-        // it by more than the threshold, so exponentials stay below 2^threshold.
-        float alpha = 1.f;
-        const bool grow = ms > m_ref + kRescaleThreshold;  // also true when m_ref == -inf
-        if (grow) {
-          alpha = fast_exp2(m_ref - ms);  // 0 when m_ref == -inf
-          m_ref = ms;
-        }
-        if (j > 0 && __any_sync(0xffffffffu, grow)) {
+        if (redo) {
+          const float ms = mx * g.scale_log2;
+          float alpha = 1.f;
+          if (ms > m_ref + kRescaleThreshold) {   // also true when m_ref == -inf
+            alpha = fast_exp2(m_ref - ms);        // 0 when m_ref == -inf
+            m_ref = ms;
+          }
           l *= alpha;
 #pragma unroll
           for (int c4 = 0; c4 < 4; ++c4) {
@@ -721,32 +830,19 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
             tc_st32(tO + c4 * 32, o);
           }
+          sum = exp_pass(m_ref == neg_inf ? 0.f : m_ref, mx, !PSA_OPTIMISTIC);
         }
-        const float m_use = (m_ref == neg_inf) ? 0.f : m_ref;
-        float sum0 = 0.f, sum1 = 0.f;
-        // probabilities in two halves of 64 keys: the first P V MMAs start while the
-        // second half of the exponentials is still being computed
-#pragma unroll
-        for (int half = 0; half < 2; ++half) {
-#pragma unroll
-          for (int c2 = 0; c2 < 2; ++c2) {
-            const int c4 = half * 2 + c2;
-            uint32_t pk[16];
-#pragma unroll
-            for (int c = 0; c < 16; ++c) {
-              const float p0 = fast_exp2(fmaf(__uint_as_float(s[c4 * 32 + 2 * c]), g.scale_log2, -m_use));
-              const float p1 = fast_exp2(fmaf(__uint_as_float(s[c4 * 32 + 2 * c + 1]), g.scale_log2, -m_use));
-              sum0 += p0;
-              sum1 += p1;
-              pk[c] = pack_bf16(p0, p1);
-            }
-            tc_st16(tS + c4 * 16, pk);
-          }
+#if PSA_SPLIT_P && PSA_OPTIMISTIC
+        if (j > 0) {  // the optimistic pass may not publish a half before it is confirmed
           tc_wait_st();
           tc_fence_before();
-          mbar_arrive(bar((half == 0 ? kBarPHalf : kBarPReady) + qi));
+          mbar_arrive(bar(kBarPHalf + qi));
         }
-        l += sum0 + sum1;
+#endif
+        l += sum;
+        tc_wait_st();
+        tc_fence_before();
+        mbar_arrive(bar(kBarPReady + qi));
       }
       if (!ok) break;
       // ---- epilogue: out = O / l, lse = ln2 * (m_ref + log2 l)
@@ -856,3 +952,4 @@ cudaError_t launch_attn(const CUtensorMap& tq, const CUtensorMap& tk, const CUte
 }
 
 }  // namespace psa
+
