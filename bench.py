@@ -172,6 +172,7 @@ def run_ours(args, w):
     from paper_2609_37001_b200 import build
     build.build()
     from paper_2609_37001_b200 import binding as B
+    from paper_2609_37001_b200 import replicas as R
     from paper_2609_37001_b200 import workloads as WL
 
     rank = int(os.environ.get("RANK", "0"))
@@ -241,10 +242,7 @@ def run_ours(args, w):
         if st != 0:
             raise SystemExit(f"device status {st} detail {hex(detail)}")
 
-        t = torch.tensor([ms_step], dtype=torch.float64, device=dev)
-        if world > 1:
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_max = float(t.item())
+        ms_max = R.max_over_ranks(ms_step, dev)
 
         extra = {}
         if rank == 0 and not args.quick:
@@ -298,10 +296,7 @@ def run_ours(args, w):
                 e2e_step()
             torch.cuda.synchronize()
             e2e_ms = 1e3 * (time.perf_counter() - t0) / ne
-            te = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
-            if world > 1:
-                dist.all_reduce(te, op=dist.ReduceOp.MAX)
-            e2e_ms = float(te.item())
+            e2e_ms = R.max_over_ranks(e2e_ms, dev)
             bytes_t = nh * L * HEAD_DIM * 2
             e2e = {"value": world * flops / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
                    "h2d_bytes_per_step": 3 * bytes_t, "d2h_bytes_per_step": bytes_t + nh * L * 4}

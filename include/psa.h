@@ -109,6 +109,13 @@ int psa_attn_fwd_host(const void* q, const void* k, const void* v, void* out, fl
  * diagnostic code naming the wait that gave up. */
 int psa_last_device_status(int32_t* detail);
 
+/* Self-test of the bounded device-side waits (no counterpart in the paper): launches a
+ * one-warp kernel that waits, with the same routine the attention kernel uses, on a barrier
+ * nothing ever arrives on.  The wait gives up after limit_ms (1..1000) and the kernel
+ * returns normally; psa_last_device_status() then reports PSA_ERR_TIMEOUT with detail
+ * 0x7e57, and the context stays usable. */
+int psa_selftest_wait_timeout(int limit_ms, void* stream);
+
 /* Measurement hook: when both are non-NULL cudaEvent_t handles, every later psa_attn_fwd
  * records `start` on its stream just before the attention kernel and `stop` just after
  * it (the planning kernel stays outside the pair).  Pass NULL, NULL to switch it off. */

@@ -64,6 +64,8 @@ def lib() -> ctypes.CDLL:
         L.psa_attn_fwd_host.argtypes = [vp] * 10 + [hp, pp, i32, i32, i32, vp]
         L.psa_last_device_status.argtypes = [ctypes.POINTER(ctypes.c_int32)]
         L.psa_shutdown.argtypes = []
+        L.psa_selftest_wait_timeout.argtypes = [i32, vp]
+        L.psa_selftest_wait_timeout.restype = ctypes.c_int
         L.psa_profile_events.argtypes = [vp, vp]
         L.psa_profile_events.restype = ctypes.c_int
         for f in (L.psa_mask_sizes, L.psa_mask_build, L.psa_attn_fwd, L.psa_attn_fwd_host,
@@ -200,6 +202,11 @@ def psa_profile_events(start: Optional[torch.cuda.Event], stop: Optional[torch.c
     a = None if start is None else ctypes.c_void_p(start.cuda_event)
     b = None if stop is None else ctypes.c_void_p(stop.cuda_event)
     _check(lib().psa_profile_events(a, b), "psa_profile_events")
+
+
+def psa_selftest_wait_timeout(limit_ms: int = 20, stream: Optional[torch.cuda.Stream] = None) -> None:
+    """Launches the bounded-wait self-test kernel (see psa.h); read the outcome with psa_last_device_status()."""
+    _check(lib().psa_selftest_wait_timeout(int(limit_ms), _stream_ptr(stream)), "psa_selftest_wait_timeout")
 
 
 def psa_launch_count() -> int:

@@ -76,14 +76,15 @@ __device__ __forceinline__ unsigned long long globaltimer_ns() {
 }
 // Bounded wait.  Returns false once the CTA-wide abort flag is set (by this or another
 // waiter); `code` names the wait for the status word.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int code) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int code,
+                                          unsigned long long limit_ns = kTimeoutNs) {
   if (mbar_try_wait(bar, parity)) return true;
   const unsigned long long t0 = globaltimer_ns();
   uint32_t n = 0;
   while (!mbar_try_wait(bar, parity)) {
     if ((++n & 255u) == 0u) {
       if (*abort_flag != 0) return false;
-      if (globaltimer_ns() - t0 > kTimeoutNs) {
+      if (globaltimer_ns() - t0 > limit_ns) {
         atomicCAS((int*)abort_flag, 0, code);
         return false;
       }
@@ -915,6 +916,29 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(*tmem_slot), "r"(512) : "memory");
   }
+}
+
+// One warp waits, with the kernel's own bounded wait, on a barrier that nothing arrives on.
+// The wait must give up after limit_ns, record PSA_ERR_TIMEOUT and return normally.
+__global__ void wait_probe_kernel(int* ws_header, unsigned long long limit_ns) {
+  __shared__ __align__(8) unsigned long long probe_bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    mbar_init(smem_u32(&probe_bar), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncwarp();
+  const bool ok = mbar_wait(smem_u32(&probe_bar), 0, &abort_flag, 0x7e57, limit_ns);
+  __syncwarp();
+  if (threadIdx.x == 0 && !ok) {
+    if (atomicCAS(ws_header + kWsStatus, 0, (int)PSA_ERR_TIMEOUT) == 0) ws_header[kWsDetail] = abort_flag;
+  }
+}
+
+cudaError_t launch_wait_probe(int* ws_header, unsigned long long limit_ns, cudaStream_t stream) {
+  wait_probe_kernel<<<1, 32, 0, stream>>>(ws_header, limit_ns);
+  return cudaGetLastError();
 }
 
 // ----------------------------------------------------------------------------- launchers

@@ -19,6 +19,7 @@ cudaError_t launch_plan(const HeadParamsArray& hp, const Geom& g, int head0, int
 cudaError_t launch_attn(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to,
                         const Geom& g, const WorkItem* items, const psa_head_params* hp_dev, int* ws_header,
                         float* lse, int n_items, int n_sms, cudaStream_t stream);
+cudaError_t launch_wait_probe(int* ws_header, unsigned long long limit_ns, cudaStream_t stream);
 }  // namespace psa
 
 namespace {
@@ -326,6 +327,23 @@ int psa_attn_fwd_host(const void* q, const void* k, const void* v, void* out, fl
   if (cudaMemcpyAsync(lse, d_lse, sizeof(float) * (size_t)prob->n_heads * L, cudaMemcpyDeviceToHost, st) != cudaSuccess)
     return PSA_ERR_CUDA;
   if (cudaStreamSynchronize(st) != cudaSuccess) return PSA_ERR_CUDA;
+  return PSA_OK;
+}
+
+int psa_selftest_wait_timeout(int limit_ms, void* stream) {
+  if (limit_ms < 1 || limit_ms > 1000) return PSA_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lock(g_mu);
+  int dev;
+  Workspace* ws;
+  int rc = device_info(&dev, &ws);
+  if (rc != PSA_OK) return rc;
+  rc = ensure_workspace(ws, 4096);
+  if (rc != PSA_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (cudaMemsetAsync(ws->base, 0, sizeof(int) * kWsHeaderWords, st) != cudaSuccess) return PSA_ERR_CUDA;
+  if (launch_wait_probe(static_cast<int*>(ws->base), 1000000ull * (unsigned long long)limit_ms, st) != cudaSuccess)
+    return PSA_ERR_CUDA;
+  ++g_launches;
   return PSA_OK;
 }
 
