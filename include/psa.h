@@ -93,6 +93,33 @@ int psa_attn_fwd(const void* q, const void* k, const void* v, void* out, float* 
                  const psa_head_params* head_params, const psa_problem* prob,
                  int T, int H, int W, void* stream);
 
+/* psa_attn_fwd for callers that must not allocate device memory (the paper has no
+ * counterpart; this is a property of the library, not of the method).
+ *
+ * Some callers cannot tolerate a cudaMalloc inside a library call: a serving loop whose
+ * device memory is entirely owned by a framework's pool, a plugin hook whose contract forbids
+ * allocation, or latency-critical code for which the device-wide synchronisation that
+ * cudaMalloc/cudaFree imply is unacceptable.  psa_attn_fwd grows a cached workspace with
+ * cudaMalloc when a larger problem arrives; this variant never does.  Its scratch (status
+ * word, scheduler ticket, per-head parameters, work order) is a fixed array of about 260 KB
+ * that is part of the library image: every GPU that loads the library holds it until exit.
+ *
+ * Same arguments, layouts and results as psa_attn_fwd, plus:
+ *   status_detail  host, optional.  NULL: the call only enqueues work on `stream`.  Non-NULL:
+ *                  the call synchronises `stream`, stores the kernel's diagnostic word there
+ *                  and returns PSA_ERR_TIMEOUT if a bounded device-side wait expired.
+ * Limits: n_heads <= 128 and n_heads * NB * ceil(slabs_per_block / 2) <= 16384 work items
+ * (Wan 2.1 14B at 1x16x16: 12,600); larger problems return PSA_ERR_CAPACITY and launch nothing.
+ * The first call on a device looks up the array's device address (with that device current);
+ * make that first call before any stream capture begins.  Every call on a device shares the
+ * array: the planning kernel clears the words that must start at zero and rewrites the rest,
+ * so back-to-back calls on one stream are fine, but calls that overlap on the GPU (different
+ * streams) race on it.  The status word of this variant is not visible to
+ * psa_last_device_status().  No cudaMalloc, cudaFree or other allocating call is made. */
+int psa_attn_fwd_noalloc(const void* q, const void* k, const void* v, void* out, float* lse,
+                         const psa_head_params* head_params, const psa_problem* prob,
+                         int T, int H, int W, void* stream, int32_t* status_detail);
+
 /* The same call for HOST tensors: copies q, k, v (host, pinned for speed) into the
  * caller's device staging buffers d_q, d_k, d_v, runs psa_attn_fwd into d_out / d_lse
  * and copies the results to out / lse (host), all on `stream`, then synchronises it.

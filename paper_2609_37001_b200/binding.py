@@ -62,6 +62,8 @@ def lib() -> ctypes.CDLL:
         L.psa_mask_build.argtypes = [hp, pp, i32, i32, i32, vp, vp, vp, ctypes.c_int64, vp]
         L.psa_attn_fwd.argtypes = [vp, vp, vp, vp, vp, hp, pp, i32, i32, i32, vp]
         L.psa_attn_fwd_host.argtypes = [vp] * 10 + [hp, pp, i32, i32, i32, vp]
+        L.psa_attn_fwd_noalloc.argtypes = [vp, vp, vp, vp, vp, hp, pp, i32, i32, i32, vp, ctypes.POINTER(ctypes.c_int32)]
+        L.psa_attn_fwd_noalloc.restype = ctypes.c_int
         L.psa_last_device_status.argtypes = [ctypes.POINTER(ctypes.c_int32)]
         L.psa_shutdown.argtypes = []
         L.psa_selftest_wait_timeout.argtypes = [i32, vp]
@@ -167,6 +169,32 @@ def psa_attn_fwd(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, head_params,
                               _params_array(head_params), ctypes.byref(prob), T, H, W, _stream_ptr(stream)),
            "psa_attn_fwd")
     return out, lse
+
+
+def psa_attn_fwd_noalloc(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, out: torch.Tensor, lse: torch.Tensor,
+                         head_params, grid: Sequence[int], tile: Sequence[int], scale: float,
+                         stream: Optional[torch.cuda.Stream] = None, check: bool = True) -> int:
+    """psa_attn_fwd through the entry point that never allocates device memory: for callers whose device
+    memory is owned by someone else's pool, or who cannot afford the device-wide synchronisation of
+    cudaMalloc.  The caller supplies ``out`` and ``lse`` (nothing is allocated here either); the library's
+    scratch is a fixed array inside the library image, so the problem must fit its limits (see psa.h).
+    With ``check`` the call synchronises the stream and raises on a device-side timeout; it returns the
+    diagnostic word."""
+    _require_cuda(q, k, v, out, lse)
+    nh, L, d = q.shape
+    T, H, W = (int(x) for x in grid)
+    if L != T * H * W or k.shape != q.shape or v.shape != q.shape or out.shape != q.shape:
+        raise ValueError("shape mismatch")
+    if q.stride() != k.stride() or q.stride() != v.stride() or q.stride() != out.stride() or q.stride(2) != 1:
+        raise ValueError("q, k, v, out must share strides with a contiguous last dimension")
+    if not lse.is_contiguous() or tuple(lse.shape) != (nh, L):
+        raise ValueError("lse must be a contiguous [heads, L] tensor")
+    prob = make_problem(nh, tile, scale, q.stride(0), q.stride(1), d)
+    detail = ctypes.c_int32(0)
+    _check(lib().psa_attn_fwd_noalloc(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), lse.data_ptr(),
+                                      _params_array(head_params), ctypes.byref(prob), T, H, W, _stream_ptr(stream),
+                                      ctypes.byref(detail) if check else None), "psa_attn_fwd_noalloc")
+    return detail.value
 
 
 def psa_attn_fwd_host(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, out: torch.Tensor, lse: torch.Tensor,

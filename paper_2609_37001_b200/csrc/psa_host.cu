@@ -165,6 +165,30 @@ int encode_map(CUtensorMap* tm, const void* base, const Geom& g, const psa_probl
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// ---- scratch of psa_attn_fwd_noalloc ------------------------------------------------------
+// Layout: 16 int32 header words (status, detail, scheduler ticket), kMaxHeads head parameter
+// records, then up to kNoAllocMaxItems work items.  It lives in every GPU that loads the
+// library, from load to exit.
+constexpr int kNoAllocMaxItems = 16384;
+constexpr size_t kNoAllocParamsOff = sizeof(int) * kWsHeaderWords;
+constexpr size_t kNoAllocItemsOff = (kNoAllocParamsOff + sizeof(psa_head_params) * kMaxHeads + 255) & ~size_t(255);
+constexpr size_t kNoAllocBytes = kNoAllocItemsOff + sizeof(WorkItem) * (size_t)kNoAllocMaxItems;
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocBytes];
+
+// Device address of the array, looked up once per device with that device current.  In host
+// code the array's name is only a handle for the runtime, never an address a kernel may use.
+void* g_noalloc_ptr[kMaxDevices] = {};
+
+int noalloc_scratch(int dev, void** ptr) {
+  if (!g_noalloc_ptr[dev]) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || p == nullptr) return PSA_ERR_CUDA;
+    g_noalloc_ptr[dev] = p;
+  }
+  *ptr = g_noalloc_ptr[dev];
+  return PSA_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -174,7 +198,7 @@ const char* psa_status_string(int status) {
     case PSA_OK: return "ok";
     case PSA_ERR_INVALID_ARG: return "invalid argument";
     case PSA_ERR_UNSUPPORTED: return "unsupported configuration";
-    case PSA_ERR_CAPACITY: return "col_idx capacity too small";
+    case PSA_ERR_CAPACITY: return "capacity exceeded (col_idx too small, or problem beyond the fixed scratch)";
     case PSA_ERR_CUDA: return "CUDA call failed";
     case PSA_ERR_TIMEOUT: return "device-side wait timed out";
     default: return "unknown status";
@@ -305,6 +329,65 @@ int psa_attn_fwd(const void* q, const void* k, const void* v, void* out, float* 
       return PSA_ERR_CUDA;
     if (g_ev_start && g_ev_stop) cudaEventRecord(g_ev_stop, st);
     ++g_launches;
+  }
+  return PSA_OK;
+}
+
+int psa_attn_fwd_noalloc(const void* q, const void* k, const void* v, void* out, float* lse,
+                         const psa_head_params* head_params, const psa_problem* prob, int T, int H, int W, void* stream,
+                         int32_t* status_detail) {
+  Geom g;
+  int rc = make_geom(prob, T, H, W, true, &g);
+  if (rc != PSA_OK) return rc;
+  if (!q || !k || !v || !out || !lse || !head_params) return PSA_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || (reinterpret_cast<uintptr_t>(lse) & 3u))
+    return PSA_ERR_INVALID_ARG;
+  if (out == q || out == k || out == v) return PSA_ERR_INVALID_ARG;
+  if (prob->stride_token < kHeadDim || (prob->stride_token % 8) != 0) return PSA_ERR_INVALID_ARG;
+  if (prob->n_heads > 1 && (prob->stride_head < kHeadDim || (prob->stride_head % 8) != 0)) return PSA_ERR_INVALID_ARG;
+  for (int h = 0; h < prob->n_heads; ++h)
+    if (!valid_params(head_params[h])) return PSA_ERR_INVALID_ARG;
+  // the fixed scratch bounds the problem: one launch worth of heads and kNoAllocMaxItems items
+  const long long n_items_ll = (long long)prob->n_heads * g.NB * g.items_per_block;
+  if (prob->n_heads > kMaxHeads || n_items_ll > kNoAllocMaxItems) return PSA_ERR_CAPACITY;
+
+  std::lock_guard<std::mutex> lock(g_mu);
+  int dev;
+  Workspace* ws;
+  rc = device_info(&dev, &ws);
+  if (rc != PSA_OK) return rc;
+  if (ws->cc_major != 10) return PSA_ERR_UNSUPPORTED;
+  rc = load_driver_entry();
+  if (rc != PSA_OK) return rc;
+  void* base = nullptr;
+  rc = noalloc_scratch(dev, &base);
+  if (rc != PSA_OK) return rc;
+  int* header = static_cast<int*>(base);
+  psa_head_params* hp_dev = reinterpret_cast<psa_head_params*>(static_cast<char*>(base) + kNoAllocParamsOff);
+  WorkItem* items = reinterpret_cast<WorkItem*>(static_cast<char*>(base) + kNoAllocItemsOff);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+
+  HeadParamsArray hp;
+  std::memset(&hp, 0, sizeof(hp));
+  for (int h = 0; h < prob->n_heads; ++h) hp.p[h] = head_params[h];
+  CUtensorMap tq, tk, tv, to;
+  if ((rc = encode_map(&tq, q, g, prob, prob->n_heads)) != PSA_OK) return rc;
+  if ((rc = encode_map(&tk, k, g, prob, prob->n_heads)) != PSA_OK) return rc;
+  if ((rc = encode_map(&tv, v, g, prob, prob->n_heads)) != PSA_OK) return rc;
+  if ((rc = encode_map(&to, out, g, prob, prob->n_heads)) != PSA_OK) return rc;
+  // The planning kernel clears the header words (status, ticket) and rewrites the parameter
+  // records and every work item of this call, so nothing of the previous call is read.
+  if (launch_plan(hp, g, 0, prob->n_heads, header, hp_dev, items, st) != cudaSuccess) return PSA_ERR_CUDA;
+  ++g_launches;
+  if (launch_attn(tq, tk, tv, to, g, items, hp_dev, header, lse, (int)n_items_ll, ws->n_sms, st) != cudaSuccess)
+    return PSA_ERR_CUDA;
+  ++g_launches;
+  if (status_detail) {
+    if (cudaStreamSynchronize(st) != cudaSuccess) return PSA_ERR_CUDA;
+    int hdr[2] = {0, 0};
+    if (cudaMemcpy(hdr, header, sizeof(hdr), cudaMemcpyDeviceToHost) != cudaSuccess) return PSA_ERR_CUDA;
+    *status_detail = hdr[1];
+    return hdr[0];
   }
   return PSA_OK;
 }
