@@ -304,11 +304,12 @@ def run_ours(args, w):
     if rank == 0:
         value = world * flops / (ms_max * 1e-3) / 1e12
         achieved = flops / (kernel_ms * 1e-3) / 1e12
-        traffic = None
-        tp = os.path.join(ROOT, "profiles", "attn_fwd_traffic.json")
+        traffic = None   # DRAM bytes per launch from the committed ncu summary of this workload
+        tp = os.path.join(ROOT, "profiles", f"attn_fwd_kernel_{w['name']}.md")
         if os.path.exists(tp):
-            with open(tp) as f:
-                traffic = json.load(f).get(w["name"])
+            for ln in open(tp):
+                if ln.startswith("traffic_bytes_per_launch:"):
+                    traffic = int(ln.split(":")[1])
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_max, "higher_is_better": True, "scaling": "weak",
