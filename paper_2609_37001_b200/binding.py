@@ -86,10 +86,20 @@ def _check(status: int, what: str) -> None:
         raise PsaError(status, what)
 
 
+_PARAMS_CACHE: dict = {}
+
+
 def _params_array(head_params: Sequence[Sequence[int]]):
-    arr = (HeadParams * len(head_params))()
-    for i, p in enumerate(head_params):
-        arr[i] = HeadParams(*[int(x) for x in p])
+    """ctypes array of the per-head parameters (memoised: repeated calls with the same heads are common)."""
+    key = tuple(tuple(int(x) for x in p) for p in head_params)
+    arr = _PARAMS_CACHE.get(key)
+    if arr is None:
+        arr = (HeadParams * len(key))()
+        for i, p in enumerate(key):
+            arr[i] = HeadParams(*p)
+        if len(_PARAMS_CACHE) > 64:
+            _PARAMS_CACHE.clear()
+        _PARAMS_CACHE[key] = arr
     return arr
 
 

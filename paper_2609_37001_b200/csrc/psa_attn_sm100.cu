@@ -219,7 +219,7 @@ __device__ __forceinline__ void exp2_poly_pair(uint64_t x2, float& p0, float& p1
   p1 = __int_as_float(__float_as_int(q1) + (__float_as_int(t1) << 23));
 }
 #ifndef PSA_EMU_PAIRS
-#define PSA_EMU_PAIRS 1   // of every 4 pairs of probabilities, this many use exp2_poly_pair
+#define PSA_EMU_PAIRS 0   // of every 4 pairs of probabilities, this many use exp2_poly_pair (0: all ex2.approx)
 #endif
 #ifndef PSA_SPLIT_P
 #define PSA_SPLIT_P 1     // publish P in two halves of 64 keys

@@ -7,12 +7,13 @@
 #include <cmath>
 #include <cstring>
 #include <mutex>
+#include <vector>
 
 #include "psa_common.cuh"
 
 namespace psa {
-cudaError_t launch_mask_build(const HeadParamsArray& hp, const Geom& g, int head0, int n_heads_here,
-                              uint8_t* block_mask, int* row_ptr, int* col_idx, int ptr_base,
+cudaError_t launch_mask_build(const HeadParamsArray& hp, const int* head_bases, const Geom& g, int n_heads_here,
+                              uint8_t* block_mask, int* row_ptr, int* col_idx, int total_nnz_through_chunk,
                               int n_sms, cudaStream_t stream, int* launches);
 cudaError_t launch_plan(const HeadParamsArray& hp, const Geom& g, int head0, int n_heads_here, int* ws_header,
                         psa_head_params* hp_dev, WorkItem* items, cudaStream_t stream);
@@ -243,11 +244,13 @@ int psa_mask_build(const psa_head_params* params, const psa_problem* prob, int T
   if (block_mask && !aligned16(block_mask)) return PSA_ERR_INVALID_ARG;
   if ((row_ptr && (reinterpret_cast<uintptr_t>(row_ptr) & 3u)) || (col_idx && (reinterpret_cast<uintptr_t>(col_idx) & 3u)))
     return PSA_ERR_INVALID_ARG;
-  long long nnz = 0;
+  // exclusive prefix of the per-head pair counts (host arithmetic, a few thousand operations)
+  std::vector<long long> base(prob->n_heads + 1, 0);
   for (int h = 0; h < prob->n_heads; ++h) {
     if (!valid_params(params[h])) return PSA_ERR_INVALID_ARG;
-    nnz += head_nnz(params[h], g);
+    base[h + 1] = base[h] + head_nnz(params[h], g);
   }
+  const long long nnz = base[prob->n_heads];
   if (nnz >= (1ll << 31) || (long long)prob->n_heads * g.NB >= (1ll << 31) - 1) return PSA_ERR_UNSUPPORTED;
   if (col_idx && col_capacity < nnz) return PSA_ERR_CAPACITY;
   int dev;
@@ -255,20 +258,20 @@ int psa_mask_build(const psa_head_params* params, const psa_problem* prob, int T
   std::lock_guard<std::mutex> lock(g_mu);
   rc = device_info(&dev, &ws);
   if (rc != PSA_OK) return rc;
-  long long ptr_base = 0;
   for (int head0 = 0; head0 < prob->n_heads; head0 += kMaxHeads) {
     const int n_here = prob->n_heads - head0 < kMaxHeads ? prob->n_heads - head0 : kMaxHeads;
     HeadParamsArray hp;
-    std::memset(&hp, 0, sizeof(hp));
-    // kernels index hp.p[head0 + h] relative to the chunk: store the chunk at its own offset
-    for (int h = 0; h < n_here; ++h) hp.p[h] = params[head0 + h];
+    int bases[kMaxHeads];
+    for (int h = 0; h < n_here; ++h) {
+      hp.p[h] = params[head0 + h];
+      bases[h] = (int)base[head0 + h];
+    }
     int launches = 0;
-    const cudaError_t e = launch_mask_build(hp, g, 0, n_here, block_mask ? block_mask + (long long)head0 * g.NB * g.NB : nullptr,
-                                            row_ptr ? row_ptr + (long long)head0 * g.NB : nullptr, col_idx, (int)ptr_base,
-                                            ws->n_sms, static_cast<cudaStream_t>(stream), &launches);
+    const cudaError_t e = launch_mask_build(hp, bases, g, n_here, block_mask ? block_mask + (long long)head0 * g.NB * g.NB : nullptr,
+                                            row_ptr ? row_ptr + (long long)head0 * g.NB : nullptr, col_idx,
+                                            (int)base[head0 + n_here], ws->n_sms, static_cast<cudaStream_t>(stream), &launches);
     g_launches += launches;
     if (e != cudaSuccess) return PSA_ERR_CUDA;
-    for (int h = 0; h < n_here; ++h) ptr_base += head_nnz(params[head0 + h], g);
   }
   return PSA_OK;
 }

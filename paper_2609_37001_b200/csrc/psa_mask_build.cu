@@ -1,145 +1,153 @@
 // psa_mask_build: block mask and GetKVBlocks index lists from the stripe parameters
 // (Algorithm 1 evaluated on block coordinates; Algorithm 2, producer side).
 // Integer work only, bound by the HBM writes of the mask bytes and the column ids.
+//
+// The two conditions of Algorithm 1 depend only on coordinate differences, so each block of
+// threads first tabulates, for its head, "does difference d attend" for every temporal and
+// every spatial difference (one modulo per table entry instead of two per mask byte).  Row
+// counts are window sums of those tables, and the block mask of a head is the Kronecker
+// product of its two axis masks, so the count of row (t', s') is cntT(t') * cntS(s') and
+// its offset in the column list has a closed form.
 #include "psa_common.cuh"
 
 namespace psa {
 
-// Row counts and their exclusive prefix sum.  The block mask of a head is the Kronecker
-// product of its temporal and spatial axis masks, so the count of row (t', s') is
-// cntT(t') * cntS(s').  One block; rows are scanned in chunks of blockDim.x.
-__global__ void __launch_bounds__(1024)
-mask_rowptr_kernel(const HeadParamsArray hp, const Geom g, int head0, int n_heads_here,
-                   int* __restrict__ row_ptr, int row_base, int ptr_base) {
-  extern __shared__ int sm[];  // [n_heads_here][Tp + Sp] axis row counts, then 1024 scan words
-  const int per_head = g.Tp + g.Sp;
-  int* cnt = sm;
-  int* scan = sm + n_heads_here * per_head;
-  for (int idx = threadIdx.x; idx < n_heads_here * per_head; idx += blockDim.x) {
-    const int h = idx / per_head, a = idx % per_head;
-    const psa_head_params p = hp.p[head0 + h];
+struct HeadBases {
+  int base[kMaxHeads];  // number of attended block pairs of all earlier heads
+};
+
+// Shared-memory tables of one head.  attT[d + Tp-1], attS[d + Sp-1] for differences d;
+// cntT[t], cntS[s] row counts per axis; preT[t], preS[s] their exclusive prefix sums.
+struct Tables {
+  uint8_t* attT;
+  uint8_t* attS;
+  int* cntT;
+  int* cntS;
+  int* preT;
+  int* preS;
+};
+
+__host__ __device__ inline size_t tables_bytes(const Geom& g) {
+  const size_t bytes = (size_t)(2 * g.Tp - 1) + (size_t)(2 * g.Sp - 1);
+  return ((bytes + 15) & ~size_t(15)) + sizeof(int) * 2 * (size_t)(g.Tp + g.Sp);
+}
+
+__device__ __forceinline__ Tables carve_tables(uint8_t* smem, const Geom& g) {
+  Tables t;
+  t.attT = smem;
+  t.attS = smem + (2 * g.Tp - 1);
+  const size_t bytes = (size_t)(2 * g.Tp - 1) + (size_t)(2 * g.Sp - 1);
+  int* ints = reinterpret_cast<int*>(smem + ((bytes + 15) & ~size_t(15)));
+  t.cntT = ints;
+  t.cntS = ints + g.Tp;
+  t.preT = t.cntS + g.Sp;
+  t.preS = t.preT + g.Tp;
+  return t;
+}
+
+// Builds the tables of one head cooperatively (whole block), ends with a barrier.
+__device__ void build_tables(const Tables& t, const psa_head_params& p, const Geom& g) {
+  for (int i = threadIdx.x; i < 2 * g.Tp - 1; i += blockDim.x) t.attT[i] = axis_attends(i - (g.Tp - 1), p.Tw, p.To, p.Ts);
+  for (int i = threadIdx.x; i < 2 * g.Sp - 1; i += blockDim.x) t.attS[i] = axis_attends(i - (g.Sp - 1), p.Sw, p.So, p.Ss);
+  __syncthreads();
+  // cnt[x] = number of key coordinates k in [0, n) with att[k - x + n-1]: a window of n entries
+  for (int x = threadIdx.x; x < g.Tp; x += blockDim.x) {
     int c = 0;
-    if (a < g.Tp) {
-      for (int k = 0; k < g.Tp; ++k) c += axis_attends(k - a, p.Tw, p.To, p.Ts);
-    } else {
-      const int s = a - g.Tp;
-      for (int k = 0; k < g.Sp; ++k) c += axis_attends(k - s, p.Sw, p.So, p.Ss);
-    }
-    cnt[idx] = c;
+    for (int k = 0; k < g.Tp; ++k) c += t.attT[k - x + g.Tp - 1];
+    t.cntT[x] = c;
+  }
+  // the spatial axis can be long: one warp per 32 coordinates, lanes stride over the window
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+  for (int x = warp; x < g.Sp; x += nwarps) {
+    int c = 0;
+    for (int k = lane; k < g.Sp; k += 32) c += t.attS[k - x + g.Sp - 1];
+    for (int off = 16; off > 0; off >>= 1) c += __shfl_xor_sync(0xffffffffu, c, off);
+    if (lane == 0) t.cntS[x] = c;
   }
   __syncthreads();
-  const int rows = n_heads_here * g.NB;
-  int carry = ptr_base;
-  for (int base = 0; base < rows; base += blockDim.x) {
-    const int r = base + threadIdx.x;
-    int c = 0;
-    if (r < rows) {
-      const int h = r / g.NB, qb = r % g.NB;
-      c = cnt[h * per_head + qb / g.Sp] * cnt[h * per_head + g.Tp + qb % g.Sp];
-    }
-    // inclusive scan over the block (Hillis-Steele in shared memory)
-    scan[threadIdx.x] = c;
-    __syncthreads();
-    for (int off = 1; off < blockDim.x; off <<= 1) {
-      int v = threadIdx.x >= off ? scan[threadIdx.x - off] : 0;
-      __syncthreads();
-      scan[threadIdx.x] += v;
-      __syncthreads();
-    }
-    if (r < rows) row_ptr[row_base + r] = carry + scan[threadIdx.x] - c;
-    const int total = scan[blockDim.x - 1];
-    __syncthreads();
-    carry += total;
+  if (threadIdx.x == 0) {
+    int acc = 0;
+    for (int x = 0; x < g.Tp; ++x) { t.preT[x] = acc; acc += t.cntT[x]; }
   }
-  if (threadIdx.x == 0) row_ptr[row_base + rows] = carry;
+  if (threadIdx.x == 32 || (blockDim.x <= 32 && threadIdx.x == 0)) {
+    int acc = 0;
+    for (int x = 0; x < g.Sp; ++x) { t.preS[x] = acc; acc += t.cntS[x]; }
+  }
+  __syncthreads();
 }
 
-// Mask bytes and column lists.  Work units are interleaved over the grid:
-//   units [0, n_chunks): 16 consecutive mask bytes each (flat over [head][qb][kb]);
-//   units [n_chunks, n_chunks + rows): one warp-wide pass over a row's key blocks, writing
-//   the attended ids in ascending order at row_ptr[row].
+// Offset of row (tq, sq) inside its head's column list, and its length.
+__device__ __forceinline__ void row_extent(const Tables& t, const Geom& g, int tq, int sq, int& offset, int& count) {
+  const int sumS = t.preS[g.Sp - 1] + t.cntS[g.Sp - 1];
+  offset = t.preT[tq] * sumS + t.cntT[tq] * t.preS[sq];
+  count = t.cntT[tq] * t.cntS[sq];
+}
+
+// One block per (group of query blocks, head); one warp per query block (= one CSR row and
+// one row of the byte mask).  Lanes cover 32 consecutive key blocks per step: coalesced mask
+// bytes, ballot-compacted ascending column ids.
 __global__ void __launch_bounds__(256)
-mask_fill_kernel(const HeadParamsArray hp, const Geom g, int head0, int n_heads_here,
-                 uint8_t* __restrict__ block_mask, const int* __restrict__ row_ptr,
-                 int* __restrict__ col_idx, int row_base) {
+mask_build_kernel(const HeadParamsArray hp, const HeadBases hb, const Geom g, int n_heads_here, int rows_per_block,
+                  uint8_t* __restrict__ block_mask, int* __restrict__ row_ptr, int* __restrict__ col_idx,
+                  int total_nnz) {
+  extern __shared__ __align__(16) uint8_t smem_tab[];
+  const int h = blockIdx.y;
+  const Tables t = carve_tables(smem_tab, g);
+  build_tables(t, hp.p[h], g);
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+  const int q0 = blockIdx.x * rows_per_block;
+  const int q1 = min(g.NB, q0 + rows_per_block);
   const long long nb2 = (long long)g.NB * g.NB;
-  const long long total_bytes = nb2 * n_heads_here;
-  const long long n_chunks = block_mask ? (total_bytes + 15) / 16 : 0;
-  const long long tid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  const long long nthreads = (long long)gridDim.x * blockDim.x;
-
-  for (long long c = tid; c < n_chunks; c += nthreads) {
-    const long long b0 = c * 16;
-    int h = (int)(b0 / nb2);
-    long long rem = b0 - (long long)h * nb2;
-    int qb = (int)(rem / g.NB), kb = (int)(rem % g.NB);
-    psa_head_params p = hp.p[head0 + h];
-    int tq = qb / g.Sp, sq = qb % g.Sp;
-    uint32_t w[4] = {0u, 0u, 0u, 0u};
-    const int n = (int)((total_bytes - b0) < 16 ? (total_bytes - b0) : 16);
-    for (int i = 0; i < n; ++i) {
-      const int tk = kb / g.Sp, sk = kb % g.Sp;
-      const uint32_t bit = axis_attends(tk - tq, p.Tw, p.To, p.Ts) && axis_attends(sk - sq, p.Sw, p.So, p.Ss);
-      w[i >> 2] |= bit << (8 * (i & 3));
-      if (++kb == g.NB) {
-        kb = 0;
-        if (++qb == g.NB) {
-          qb = 0;
-          ++h;
-          if (h < n_heads_here) p = hp.p[head0 + h];
-        }
-        tq = qb / g.Sp;
-        sq = qb % g.Sp;
-      }
-    }
-    uint8_t* dst = block_mask + (long long)head0 * nb2 + b0;
-    if (n == 16) {
-      *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
-    } else {
-      for (int i = 0; i < n; ++i) dst[i] = (uint8_t)(w[i >> 2] >> (8 * (i & 3)));
-    }
-  }
-
-  if (col_idx == nullptr) return;
-  const int lane = threadIdx.x & 31;
-  const long long warp = tid >> 5, nwarps = nthreads >> 5;
-  const int rows = n_heads_here * g.NB;
-  for (long long r = warp; r < rows; r += nwarps) {
-    const int h = (int)(r / g.NB), qb = (int)(r % g.NB);
-    const psa_head_params p = hp.p[head0 + h];
+  for (int qb = q0 + warp; qb < q1; qb += nwarps) {
     const int tq = qb / g.Sp, sq = qb % g.Sp;
-    int pos = row_ptr[row_base + r];
+    int offset, count;
+    row_extent(t, g, tq, sq, offset, count);
+    int pos = hb.base[h] + offset;
+    if (row_ptr && lane == 0) row_ptr[(long long)h * g.NB + qb] = pos;
+    uint8_t* mrow = block_mask ? block_mask + (long long)h * nb2 + (long long)qb * g.NB : nullptr;
+    if (mrow == nullptr && col_idx == nullptr) continue;
+    const uint8_t* aT = t.attT + (g.Tp - 1 - tq);
+    const uint8_t* aS = t.attS + (g.Sp - 1 - sq);
+    int tk = lane / g.Sp, sk = lane % g.Sp;       // coordinates of key block `lane`
+    const int dt = 32 / g.Sp, ds = 32 % g.Sp;     // advance of 32 key blocks
     for (int base = 0; base < g.NB; base += 32) {
       const int kb = base + lane;
-      bool att = false;
-      if (kb < g.NB) {
-        const int tk = kb / g.Sp, sk = kb % g.Sp;
-        att = axis_attends(tk - tq, p.Tw, p.To, p.Ts) && axis_attends(sk - sq, p.Sw, p.So, p.Ss);
+      const bool att = kb < g.NB && aT[tk] && aS[sk];
+      if (mrow && kb < g.NB) mrow[kb] = att ? 1 : 0;
+      if (col_idx) {
+        const unsigned m = __ballot_sync(0xffffffffu, att);
+        if (att) col_idx[pos + __popc(m & ((1u << lane) - 1u))] = kb;
+        pos += __popc(m);
       }
-      const unsigned m = __ballot_sync(0xffffffffu, att);
-      if (att) col_idx[pos + __popc(m & ((1u << lane) - 1u))] = kb;
-      pos += __popc(m);
+      tk += dt;
+      sk += ds;
+      if (sk >= g.Sp) { sk -= g.Sp; ++tk; }
     }
   }
+  if (row_ptr && blockIdx.x == 0 && h == n_heads_here - 1 && threadIdx.x == 0)
+    row_ptr[(long long)n_heads_here * g.NB] = total_nnz;
 }
 
-cudaError_t launch_mask_build(const HeadParamsArray& hp, const Geom& g, int head0, int n_heads_here,
-                              uint8_t* block_mask, int* row_ptr, int* col_idx, int ptr_base,
+cudaError_t launch_mask_build(const HeadParamsArray& hp, const int* head_bases, const Geom& g, int n_heads_here,
+                              uint8_t* block_mask, int* row_ptr, int* col_idx, int total_nnz_through_chunk,
                               int n_sms, cudaStream_t stream, int* launches) {
-  const int row_base = head0 * g.NB;
-  if (row_ptr) {
-    const size_t smem = sizeof(int) * ((size_t)n_heads_here * (g.Tp + g.Sp) + 1024);
-    if (smem > 48 * 1024) {
-      cudaError_t e = cudaFuncSetAttribute(mask_rowptr_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-      if (e != cudaSuccess) return e;
-    }
-    mask_rowptr_kernel<<<1, 1024, smem, stream>>>(hp, g, head0, n_heads_here, row_ptr, row_base, ptr_base);
-    ++*launches;
+  HeadBases hb;
+  for (int h = 0; h < kMaxHeads; ++h) hb.base[h] = h < n_heads_here ? head_bases[h] : 0;
+  const size_t smem = tables_bytes(g);
+  if (smem > 48 * 1024) {
+    cudaError_t e = cudaFuncSetAttribute(mask_build_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
   }
-  if (block_mask || col_idx) {
-    mask_fill_kernel<<<n_sms * 8, 256, 0, stream>>>(hp, g, head0, n_heads_here, block_mask, row_ptr, col_idx, row_base);
-    ++*launches;
-  }
+  // enough blocks per head to fill the machine about twice, at least 8 rows (one per warp) each
+  int blocks_per_head = (2 * n_sms + n_heads_here - 1) / n_heads_here;
+  if (blocks_per_head < 1) blocks_per_head = 1;
+  int rows_per_block = (g.NB + blocks_per_head - 1) / blocks_per_head;
+  if (rows_per_block < 8) rows_per_block = 8;
+  blocks_per_head = (g.NB + rows_per_block - 1) / rows_per_block;
+  dim3 grid(blocks_per_head, n_heads_here);
+  mask_build_kernel<<<grid, 256, smem, stream>>>(hp, hb, g, n_heads_here, rows_per_block, block_mask, row_ptr, col_idx,
+                                                 total_nnz_through_chunk);
+  ++*launches;
   return cudaGetLastError();
 }
 
