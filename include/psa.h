@@ -40,7 +40,7 @@ extern "C" {
 typedef enum {
   PSA_OK = 0,
   PSA_ERR_INVALID_ARG = -1, /* null/misaligned pointer, non-positive extent, bad parameter   */
-  PSA_ERR_UNSUPPORTED = -2, /* head_dim != 128, tile token count not 128/256/384, not sm_100  */
+  PSA_ERR_UNSUPPORTED = -2, /* head_dim != 128, unsupported tile shape, not sm_100             */
   PSA_ERR_CAPACITY = -3,    /* col_capacity < nnz                                             */
   PSA_ERR_CUDA = -4,        /* a CUDA runtime/driver call failed                              */
   PSA_ERR_TIMEOUT = -5      /* a bounded device-side wait expired (see psa_last_device_status) */
@@ -50,8 +50,11 @@ typedef enum {
  * mean an infinite stride.  Valid: Tw, Sw >= 1; Ts, Ss >= 0; |To|, |So| < 2^30. */
 typedef struct { int32_t Tw, To, Ts, Sw, So, Ss; } psa_head_params;
 
-/* Mask block (PSABlock) extents in tokens.  For psa_attn_fwd bt*bh*bw must be 128, 256
- * or 384 and split into 128-token slabs along its outermost non-unit axis. */
+/* Mask block (PSABlock) extents in tokens.  psa_attn_fwd splits a block into compute slabs
+ * along its outermost axis of extent > 1: slabs of exactly 128 tokens plus a last slab of
+ * 128, 112, 96 or 64 tokens, at most three slabs (128 <= bt*bh*bw <= 384).  Examples:
+ * 1x16x16 = 128+128, 3x8x16 = 3 x 128, 1x15x16 = 128+112 (tiles a 45-row grid without
+ * padding).  Other shapes return PSA_ERR_UNSUPPORTED. */
 typedef struct { int32_t bt, bh, bw; } psa_tile;
 
 typedef struct {

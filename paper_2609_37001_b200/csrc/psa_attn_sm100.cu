@@ -159,6 +159,20 @@ __device__ __forceinline__ void tc_st32(uint32_t addr, const uint32_t* r) {
         "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
       : "memory");
 }
+__device__ __forceinline__ void tc_ld16(uint32_t addr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(addr) : "memory");
+}
+__device__ __forceinline__ void tc_st8(uint32_t addr, const uint32_t* r) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+      ::"r"(addr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+      : "memory");
+}
 __device__ __forceinline__ void tc_st16(uint32_t addr, const uint32_t* r) {
   asm volatile(
       "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
@@ -224,9 +238,7 @@ __device__ __forceinline__ void exp2_poly_pair(uint64_t x2, float& p0, float& p1
 #ifndef PSA_SPLIT_P
 #define PSA_SPLIT_P 1     // publish P in two halves of 64 keys
 #endif
-#ifndef PSA_OPTIMISTIC
-#define PSA_OPTIMISTIC 0  // exponentiate with the running maximum before the slab maximum is known
-#endif
+
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
@@ -246,9 +258,9 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
   d |= 2ull << 61;  // 128-byte swizzle
   return d;
 }
-// Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = 128; A is K-major.
-__host__ __device__ constexpr uint32_t instr_desc(bool b_mn_major) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+// Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N columns (multiple of 16); A is K-major.
+__host__ __device__ constexpr uint32_t instr_desc(bool b_mn_major, uint32_t n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((n >> 3) << 17) | ((128u >> 4) << 24);
 }
 // One elected lane of a converged warp (keeps the branch warp-uniform for the compiler).
 __device__ __forceinline__ bool elect_one() {
@@ -312,6 +324,22 @@ struct AttnParams {
   int n_items;
 };
 
+struct TensorMaps {
+  CUtensorMap q[2], k[2], v[2], o[2];  // [0]: full 128-token slab box, [1]: a block's last slab
+};
+
+// Extents and token count of slab `sub` of a block; `last` selects the tensor-map set.
+__device__ __forceinline__ void slab_shape(const Geom& g, int sub, int& et, int& eh, int& ew, int& ntok, int& last) {
+  last = (sub == g.n_sub - 1) ? 1 : 0;
+  et = g.ct; eh = g.ch; ew = g.cw;
+  if (last) {
+    if (g.sub_axis == 0) et = g.c_last;
+    else if (g.sub_axis == 1) eh = g.c_last;
+    else ew = g.c_last;
+  }
+  ntok = last ? g.n_last : kSlabTokens;
+}
+
 __device__ __forceinline__ void slab_origin(const Geom& g, int qb, int sub, int& t0, int& h0, int& w0) {
   const int tb = qb / g.Sp, sb = qb % g.Sp;
   t0 = tb * g.bt;
@@ -330,10 +358,112 @@ __device__ __forceinline__ uint32_t desc_lo(uint32_t addr, uint32_t lbo_bytes) {
 }
 __device__ __forceinline__ uint64_t make_desc(uint32_t lo) { return ((uint64_t)kDescHi << 32) | lo; }
 
+// Online-softmax step of one query row (one thread) for one key slab of NK keys.
+//   tS: TMEM address of the row's scores (fp32, NK columns); the bf16 probabilities are written
+//       back over the first NK/2 columns.  tO: the row's output accumulator (128 fp32 columns).
+//   meta: [0] != 0 marks a slab with padded key positions, [1..4] = validity bits of its keys.
+//   m_ref / l: running reference maximum (scaled log2 domain) and running sum.
+// The reference maximum is lazy: it moves only when the slab's maximum exceeds it by more than
+// kRescaleThreshold, so exponentials stay below 2^threshold and O is rarely rescaled.
+template <int NK>
+__device__ __forceinline__ void softmax_slab(uint32_t tS, uint32_t tO, const uint32_t* meta, bool first,
+                                             float scale_log2, float& m_ref, float& l, uint32_t bar_half,
+                                             uint32_t bar_ready) {
+  constexpr int NFULL = NK / 32, REM = NK % 32;
+  static_assert(NK % 16 == 0 && NK >= 64 && NK <= 128 && (REM == 0 || REM == 16), "unsupported slab width");
+  const float neg_inf = __int_as_float(0xff800000);
+  uint32_t s[NK];  // raw scores of this row (fp32 bit patterns), kept in registers
+#pragma unroll
+  for (int c4 = 0; c4 < NFULL; ++c4) tc_ld32(tS + c4 * 32, s + c4 * 32);
+  if (REM) tc_ld16(tS + NFULL * 32, s + NFULL * 32);
+  tc_wait_ld();
+  if (meta[0] != 0u) {  // 3D-padding: padded key positions score -inf
+    const uint32_t v[4] = {meta[1], meta[2], meta[3], meta[4]};
+#pragma unroll
+    for (int c = 0; c < NK; ++c)
+      if (!((v[c >> 5] >> (c & 31)) & 1u)) s[c] = 0xff800000u;
+  }
+  float a0 = neg_inf, a1 = neg_inf, a2 = neg_inf, a3 = neg_inf;
+#pragma unroll
+  for (int c = 0; c < NK; c += 8) {
+    a0 = max3(a0, __uint_as_float(s[c]), __uint_as_float(s[c + 1]));
+    a1 = max3(a1, __uint_as_float(s[c + 2]), __uint_as_float(s[c + 3]));
+    a2 = max3(a2, __uint_as_float(s[c + 4]), __uint_as_float(s[c + 5]));
+    a3 = max3(a3, __uint_as_float(s[c + 6]), __uint_as_float(s[c + 7]));
+  }
+  const float ms = fmaxf(fmaxf(a0, a1), fmaxf(a2, a3)) * scale_log2;
+  if (first) {
+    m_ref = ms;  // first slab of the item: nothing accumulated yet
+  } else {
+    float alpha = 1.f;
+    const bool grow = ms > m_ref + kRescaleThreshold;  // also true when m_ref == -inf
+    if (grow) {
+      alpha = fast_exp2(m_ref - ms);  // 0 when m_ref == -inf
+      m_ref = ms;
+    }
+    if (__any_sync(0xffffffffu, grow)) {
+      l *= alpha;
+#pragma unroll
+      for (int c4 = 0; c4 < 4; ++c4) {
+        uint32_t o[32];
+        tc_ld32(tO + c4 * 32, o);
+        tc_wait_ld();
+#pragma unroll
+        for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
+        tc_st32(tO + c4 * 32, o);
+      }
+    }
+  }
+  const float m_use = (m_ref == neg_inf) ? 0.f : m_ref;
+  const uint64_t sc2 = pack2(scale_log2, scale_log2), negm2 = pack2(-m_use, -m_use);
+  uint64_t sum2 = pack2(0.f, 0.f);
+  // probabilities exp2(scale*s - m_use), bf16, written over the scores in chunks of 32 keys
+  auto exp_chunk = [&](int base, int npairs, uint32_t* pk) {
+#pragma unroll
+    for (int c = 0; c < 16; ++c) {
+      if (c >= npairs) break;
+      const uint64_t x2 = fma2(pack2(__uint_as_float(s[base + 2 * c]), __uint_as_float(s[base + 2 * c + 1])), sc2, negm2);
+      float p0, p1;
+      if ((c & 3) < PSA_EMU_PAIRS) {
+        exp2_poly_pair(x2, p0, p1);
+      } else {
+        float x0, x1;
+        unpack2(x2, x0, x1);
+        p0 = fast_exp2(x0);
+        p1 = fast_exp2(x1);
+      }
+      sum2 = add2(sum2, pack2(p0, p1));
+      pk[c] = pack_bf16(p0, p1);
+    }
+  };
+#pragma unroll
+  for (int c4 = 0; c4 < NFULL; ++c4) {
+    uint32_t pk[16];
+    exp_chunk(c4 * 32, 16, pk);
+    tc_st16(tS + c4 * 16, pk);
+#if PSA_SPLIT_P
+    if (c4 == 1) {  // the first 64 keys are final: their P V MMAs may start
+      tc_wait_st();
+      tc_fence_before();
+      mbar_arrive(bar_half);
+    }
+#endif
+  }
+  if (REM) {
+    uint32_t pk[16];
+    exp_chunk(NFULL * 32, 8, pk);
+    tc_st8(tS + NFULL * 16, pk);
+  }
+  float sum0, sum1;
+  unpack2(sum2, sum0, sum1);
+  l += sum0 + sum1;
+  tc_wait_st();
+  tc_fence_before();
+  mbar_arrive(bar_ready);
+}
+
 __global__ void __launch_bounds__(kThreads, 1)
-attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o,
-                const AttnParams prm) {
+attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const uint32_t sbase = smem_u32(smem);
@@ -348,6 +478,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + kOffMisc);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kOffMisc + 4);
 
+  // A short query slab leaves its last rows of the Q buffer unwritten; keep them finite.
+  for (uint32_t off = threadIdx.x * 16u; off < 2u * kSlabBytes; off += kThreads * 16u)
+    *reinterpret_cast<uint4*>(smem + kOffQ + off) = make_uint4(0u, 0u, 0u, 0u);
+  fence_async_smem();
   if (threadIdx.x == 0) {
     *abort_flag = 0;
     for (int i = 0; i < 2; ++i) {
@@ -448,12 +582,13 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         ok = mbar_wait_warp(bar(kBarQEmpty + i), (itq & 1u) ^ 1u, abort_flag, 0x100 + i);
         if (!ok) break;
         if (lane == 0) {
-          int t0, h0, w0;
+          int t0, h0, w0, et, eh, ew, ntok, last;
           slab_origin(g, qb, sub0 + i, t0, h0, w0);
+          slab_shape(g, sub0 + i, et, eh, ew, ntok, last);
           const uint32_t dst = sbase + kOffQ + (uint32_t)i * kSlabBytes;
-          mbar_expect_tx(bar(kBarQFull + i), kSlabBytes);
-          tma_load_5d(dst, &tm_q, bar(kBarQFull + i), 0, w0, h0, t0, head);
-          tma_load_5d(dst + kHalfBytes, &tm_q, bar(kBarQFull + i), 64, w0, h0, t0, head);
+          mbar_expect_tx(bar(kBarQFull + i), (uint32_t)ntok * 256u);
+          tma_load_5d(dst, &tms.q[last], bar(kBarQFull + i), 0, w0, h0, t0, head);
+          tma_load_5d(dst + kHalfBytes, &tms.q[last], bar(kBarQFull + i), 64, w0, h0, t0, head);
         }
         if (i == 0) ++it_q0; else ++it_q1;
       }
@@ -461,6 +596,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       // key / value slabs in ascending key-block id
       bool have_prev = false;
       int pt0 = 0, ph0 = 0, pw0 = 0;  // origin of the previous slab (its V is still to be loaded)
+      int plast = 0, pntok = kSlabTokens;
       for (int tw = 0; ok && tw < g.Tp; tw += 32) {
         uint32_t mt = maskT[tw >> 5];
         while (ok && mt) {
@@ -473,21 +609,22 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
               ms &= ms - 1;
               const int kb = tk * g.Sp + sk;
               for (int sub = 0; ok && sub < g.n_sub; ++sub) {
-                int t0, h0, w0;
+                int t0, h0, w0, et, eh, ew, ntok, last;
                 slab_origin(g, kb, sub, t0, h0, w0);
-                // validity of the slab's 128 key positions (3D-padding): bit c of word c/32
-                const bool edge = (t0 + g.ct > g.T) || (h0 + g.ch > g.H) || (w0 + g.cw > g.W);
+                slab_shape(g, sub, et, eh, ew, ntok, last);
+                // validity of the slab's key positions (3D-padding): bit c of word c/32
+                const bool edge = (t0 + et > g.T) || (h0 + eh > g.H) || (w0 + ew > g.W);
                 uint32_t vw0 = 0xffffffffu, vw1 = 0xffffffffu, vw2 = 0xffffffffu, vw3 = 0xffffffffu;
                 if (edge) {
-                  const int chw = g.cw * g.ch;
+                  const int ehw = ew * eh;
                   int c = lane;
-                  vw0 = __ballot_sync(0xffffffffu, (t0 + c / chw < g.T) && (h0 + (c / g.cw) % g.ch < g.H) && (w0 + c % g.cw < g.W));
+                  vw0 = __ballot_sync(0xffffffffu, (t0 + c / ehw < g.T) && (h0 + (c / ew) % eh < g.H) && (w0 + c % ew < g.W));
                   c += 32;
-                  vw1 = __ballot_sync(0xffffffffu, (t0 + c / chw < g.T) && (h0 + (c / g.cw) % g.ch < g.H) && (w0 + c % g.cw < g.W));
+                  vw1 = __ballot_sync(0xffffffffu, (t0 + c / ehw < g.T) && (h0 + (c / ew) % eh < g.H) && (w0 + c % ew < g.W));
                   c += 32;
-                  vw2 = __ballot_sync(0xffffffffu, (t0 + c / chw < g.T) && (h0 + (c / g.cw) % g.ch < g.H) && (w0 + c % g.cw < g.W));
+                  vw2 = __ballot_sync(0xffffffffu, (t0 + c / ehw < g.T) && (h0 + (c / ew) % eh < g.H) && (w0 + c % ew < g.W));
                   c += 32;
-                  vw3 = __ballot_sync(0xffffffffu, (t0 + c / chw < g.T) && (h0 + (c / g.cw) % g.ch < g.H) && (w0 + c % g.cw < g.W));
+                  vw3 = __ballot_sync(0xffffffffu, (t0 + c / ehw < g.T) && (h0 + (c / ew) % eh < g.H) && (w0 + c % ew < g.W));
                 }
                 // slots: [V of the previous slab,] K of this slab
                 const uint32_t v_slot = tile_g % kNumSlots, v_use = tile_g / kNumSlots;
@@ -504,16 +641,18 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                   m[0] = edge ? 1u : 0u;
                   m[1] = vw0; m[2] = vw1; m[3] = vw2; m[4] = vw3;
                   const uint32_t pb = bar(kBarPairFull + pair_g % kNumPairBars);
-                  mbar_expect_tx(pb, have_prev ? 2u * kSlabBytes : kSlabBytes);
+                  mbar_expect_tx(pb, (uint32_t)((have_prev ? pntok : 0) + ntok) * 256u);
                   if (have_prev) {
                     const uint32_t dv = sbase + kOffRing + v_slot * kSlabBytes;
-                    tma_load_5d(dv, &tm_v, pb, 0, pw0, ph0, pt0, head);
-                    tma_load_5d(dv + kHalfBytes, &tm_v, pb, 64, pw0, ph0, pt0, head);
+                    tma_load_5d(dv, &tms.v[plast], pb, 0, pw0, ph0, pt0, head);
+                    tma_load_5d(dv + kHalfBytes, &tms.v[plast], pb, 64, pw0, ph0, pt0, head);
                   }
                   const uint32_t dk = sbase + kOffRing + k_slot * kSlabBytes;
-                  tma_load_5d(dk, &tm_k, pb, 0, w0, h0, t0, head);
-                  tma_load_5d(dk + kHalfBytes, &tm_k, pb, 64, w0, h0, t0, head);
+                  tma_load_5d(dk, &tms.k[last], pb, 0, w0, h0, t0, head);
+                  tma_load_5d(dk + kHalfBytes, &tms.k[last], pb, 64, w0, h0, t0, head);
                 }
+                plast = last;
+                pntok = ntok;
                 tile_g = k_tile + 1;
                 ++pair_g;
                 ++kv_g;
@@ -530,10 +669,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         if (!ok) break;
         if (lane == 0) {
           const uint32_t pb = bar(kBarPairFull + pair_g % kNumPairBars);
-          mbar_expect_tx(pb, kSlabBytes);
+          mbar_expect_tx(pb, (uint32_t)pntok * 256u);
           const uint32_t dv = sbase + kOffRing + v_slot * kSlabBytes;
-          tma_load_5d(dv, &tm_v, pb, 0, pw0, ph0, pt0, head);
-          tma_load_5d(dv + kHalfBytes, &tm_v, pb, 64, pw0, ph0, pt0, head);
+          tma_load_5d(dv, &tms.v[plast], pb, 0, pw0, ph0, pt0, head);
+          tma_load_5d(dv + kHalfBytes, &tms.v[plast], pb, 64, pw0, ph0, pt0, head);
         }
         ++tile_g;
         ++pair_g;
@@ -563,8 +702,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     __syncwarp();
   } else if (warp == 9) {
     // ======================================================================= MMA warp
-    constexpr uint32_t kIdescQK = instr_desc(false);
-    constexpr uint32_t kIdescPV = instr_desc(true);
+    constexpr uint32_t kIdescPV = instr_desc(true, 128);  // N = head_dim
     uint32_t tile_g = 0, pair_g = 0;
     uint32_t it_q0 = 0, it_q1 = 0;
     uint32_t cnt_s0 = 0, cnt_s1 = 0;  // P_i tiles consumed so far
@@ -575,23 +713,26 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     constexpr uint32_t kSlabStep = kSlabBytes >> 4;  // descriptor address units per slab
 
     // S_i = Q_i K^T over head_dim = 128: 8 MMAs of K = 16; both operands K-major, SW128.
-    auto issue_qk = [&](int i, uint32_t kslot) {
+    // nk = keys of the slab (N of the instruction): 128, or fewer for a block's last slab.
+    auto issue_qk = [&](int i, uint32_t kslot, int nk) {
       const uint32_t a0 = q_lo + (uint32_t)i * kSlabStep, b0 = ring_lo_k + kslot * kSlabStep;
+      const uint32_t idesc = instr_desc(false, (uint32_t)nk);
 #pragma unroll
       for (int kk = 0; kk < 8; ++kk) {
         const uint32_t off = (uint32_t)(kk >> 2) * (kHalfBytes >> 4) + (uint32_t)(kk & 3) * 2u;
-        tc_mma_ss(tmem + (uint32_t)i * 128u, make_desc(a0 + off), make_desc(b0 + off), kIdescQK, kk > 0 ? 1u : 0u);
+        tc_mma_ss(tmem + (uint32_t)i * 128u, make_desc(a0 + off), make_desc(b0 + off), idesc, kk > 0 ? 1u : 0u);
       }
     };
     // O_i (+)= P_i V over 128 keys: 8 MMAs of K = 16; A = bf16 P in TMEM (8 columns per
     // step), B = V slab as loaded (keys x head_dim, head_dim contiguous) = MN-major SW128:
     // 16 keys advance 2048 bytes, the second 64 columns of head_dim sit one half slab
     // further (leading byte offset).
-    auto issue_pv_half = [&](int i, uint32_t vslot, int half, bool accumulate) {
+    auto issue_pv_half = [&](int i, uint32_t vslot, int half, bool accumulate, int nk) {
       const uint32_t b0 = ring_lo_v + vslot * kSlabStep;
 #pragma unroll
       for (int k4 = 0; k4 < 4; ++k4) {
         const int kk = half * 4 + k4;
+        if (kk * 16 >= nk) break;   // a short slab has fewer 16-key steps
         tc_mma_ts(tmem + 256u + (uint32_t)i * 128u, tmem + (uint32_t)i * 128u + (uint32_t)kk * 8u,
                   make_desc(b0 + (uint32_t)kk * (2048u >> 4)), kIdescPV, (accumulate || kk > 0) ? 1u : 0u);
       }
@@ -626,7 +767,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 #pragma unroll
             for (int i = 0; i < 2; ++i) {
               if (i < nq) {
-                issue_qk(i, slot);
+                issue_qk(i, slot, g.n_sub == 1 ? g.n_last : kSlabTokens);
                 tc_commit(bar(kBarSFull + i));
               }
             }
@@ -634,7 +775,11 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           }
           __syncwarp();
         }
+        int sub = 0;  // slab index of key slab j inside its block
         for (int j = 0; ok && j < n_kv; ++j) {
+          const int nk_cur = (sub == g.n_sub - 1) ? g.n_last : kSlabTokens;
+          sub = (sub + 1 == g.n_sub) ? 0 : sub + 1;
+          const int nk_next = (sub == g.n_sub - 1) ? g.n_last : kSlabTokens;
           // V_j and (unless this is the last slab) K_{j+1} arrive under one barrier
           ok = mbar_wait_warp(bar(kBarPairFull + pair_g % kNumPairBars), (pair_g / kNumPairBars) & 1u, abort_flag, 0x211);
           if (!ok) break;
@@ -651,7 +796,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             ok = mbar_wait_warp(bar(kBarPHalf + i), cs & 1u, abort_flag, 0x224 + i);
             if (!ok) break;
             tc_fence_after();
-            if (elect_one()) issue_pv_half(i, vslot, 0, j > 0);
+            if (elect_one()) issue_pv_half(i, vslot, 0, j > 0, nk_cur);
 #endif
             ok = mbar_wait_warp(bar(kBarPReady + i), cs & 1u, abort_flag, 0x220 + i);
             if (!ok) break;
@@ -659,14 +804,14 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             tc_fence_after();
             if (elect_one()) {
 #if PSA_SPLIT_P
-              issue_pv_half(i, vslot, 1, true);
+              issue_pv_half(i, vslot, 1, true, nk_cur);
 #else
-              issue_pv_half(i, vslot, 0, j > 0);
-              issue_pv_half(i, vslot, 1, true);
+              issue_pv_half(i, vslot, 0, j > 0, nk_cur);
+              issue_pv_half(i, vslot, 1, true, nk_cur);
 #endif
               if (i == nq - 1) tc_commit(bar(kBarSlotEmpty + vslot));
               if (more) {
-                issue_qk(i, kslot);
+                issue_qk(i, kslot, nk_next);
                 tc_commit(bar(kBarSFull + i));
                 if (i == nq - 1) tc_commit(bar(kBarSlotEmpty + kslot));
               } else {
@@ -699,7 +844,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     uint32_t it_q = 0, cnt_s = 0, kv_g = 0;
     bool ok = true;
     const float neg_inf = __int_as_float(0xff800000);
-    const uint64_t sc2 = pack2(g.scale_log2, g.scale_log2);
 
     for (uint32_t n = 0; ok; ++n) {
       WorkItem wi;
@@ -712,138 +856,20 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       }
       float m_ref = neg_inf;  // running reference maximum, scaled log2 domain
       float l = 0.f;          // running sum of exp2(s - m_ref)
+      int ksub = 0;           // slab index of key slab j inside its block
       for (int j = 0; ok && j < n_kv; ++j, ++kv_g) {
+        const int nk = (ksub == g.n_sub - 1) ? g.n_last : kSlabTokens;
+        ksub = (ksub + 1 == g.n_sub) ? 0 : ksub + 1;
         ok = mbar_wait_warp(bar(kBarSFull + qi), cnt_s & 1u, abort_flag, 0x300 + qi);
         if (!ok) break;
         ++cnt_s;
         tc_fence_after();
-        uint32_t s[128];  // raw scores of this row (fp32 bit patterns), kept in registers
-        tc_ld32(tS + 0, s + 0);
-        tc_ld32(tS + 32, s + 32);
-        tc_ld32(tS + 64, s + 64);
-        tc_ld32(tS + 96, s + 96);
-        tc_wait_ld();
         const uint32_t* m = meta + (kv_g % kMetaRing) * 8;
-        if (m[0] != 0u) {  // 3D-padding: padded key positions score -inf
-          const uint32_t v0 = m[1], v1 = m[2], v2 = m[3], v3 = m[4];
-#pragma unroll
-          for (int c = 0; c < 32; ++c) {
-            if (!((v0 >> c) & 1u)) s[c] = 0xff800000u;
-            if (!((v1 >> c) & 1u)) s[32 + c] = 0xff800000u;
-            if (!((v2 >> c) & 1u)) s[64 + c] = 0xff800000u;
-            if (!((v3 >> c) & 1u)) s[96 + c] = 0xff800000u;
-          }
-        }
-        // One pass over the row: probabilities exp2(scale*s - m_use) are written to TMEM as
-        // bf16 while the row maximum is gathered on the side.  Returns the row sum.
-        auto exp_pass = [&](float m_use, float& row_max, bool signal_half) -> float {
-          const uint64_t negm2 = pack2(-m_use, -m_use);
-          uint64_t sum2 = pack2(0.f, 0.f);
-          float mx0 = neg_inf, mx1 = neg_inf, mx2 = neg_inf, mx3 = neg_inf;
-#pragma unroll
-          for (int c4 = 0; c4 < 4; ++c4) {
-            uint32_t pk[16];
-#pragma unroll
-            for (int c = 0; c < 16; ++c) {
-              const float s0 = __uint_as_float(s[c4 * 32 + 2 * c]), s1 = __uint_as_float(s[c4 * 32 + 2 * c + 1]);
-              if ((c & 3) == 0) mx0 = max3(mx0, s0, s1);
-              else if ((c & 3) == 1) mx1 = max3(mx1, s0, s1);
-              else if ((c & 3) == 2) mx2 = max3(mx2, s0, s1);
-              else mx3 = max3(mx3, s0, s1);
-              const uint64_t x2 = fma2(pack2(s0, s1), sc2, negm2);
-              float p0, p1;
-              if ((c & 3) < PSA_EMU_PAIRS) {
-                exp2_poly_pair(x2, p0, p1);
-              } else {
-                float x0, x1;
-                unpack2(x2, x0, x1);
-                p0 = fast_exp2(x0);
-                p1 = fast_exp2(x1);
-              }
-              sum2 = add2(sum2, pack2(p0, p1));
-              pk[c] = pack_bf16(p0, p1);
-            }
-            tc_st16(tS + c4 * 16, pk);
-#if PSA_SPLIT_P
-            if (c4 == 1 && signal_half) {  // first 64 keys are final: their P V MMAs may start
-              tc_wait_st();
-              tc_fence_before();
-              mbar_arrive(bar(kBarPHalf + qi));
-            }
-#endif
-          }
-          row_max = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
-          float sum0, sum1;
-          unpack2(sum2, sum0, sum1);
-          return sum0 + sum1;
-        };
-        float sum, mx;
-        bool redo;
-        if (j == 0) {
-          // first slab of the item: the reference maximum is the row maximum itself
-          float a0 = neg_inf, a1 = neg_inf, a2 = neg_inf, a3 = neg_inf;
-#pragma unroll
-          for (int c = 0; c < 128; c += 8) {
-            a0 = max3(a0, __uint_as_float(s[c]), __uint_as_float(s[c + 1]));
-            a1 = max3(a1, __uint_as_float(s[c + 2]), __uint_as_float(s[c + 3]));
-            a2 = max3(a2, __uint_as_float(s[c + 4]), __uint_as_float(s[c + 5]));
-            a3 = max3(a3, __uint_as_float(s[c + 6]), __uint_as_float(s[c + 7]));
-          }
-          m_ref = fmaxf(fmaxf(a0, a1), fmaxf(a2, a3)) * g.scale_log2;
-          sum = exp_pass(m_ref == neg_inf ? 0.f : m_ref, mx, true);
-          redo = false;
-        } else {
-#if PSA_OPTIMISTIC
-          // Optimistic pass with the running reference maximum: exponentials start right
-          // after the load instead of after a full max reduction.  The reference only has to
-          // keep exp2 bounded; it moves (lazy rescale) when the slab's maximum exceeds it by
-          // more than the threshold, which is detected here and repaired below.
-          sum = exp_pass(m_ref == neg_inf ? 0.f : m_ref, mx, false);
-          redo = __any_sync(0xffffffffu, mx * g.scale_log2 > m_ref + kRescaleThreshold);
-#else
-          float a0 = neg_inf, a1 = neg_inf, a2 = neg_inf, a3 = neg_inf;
-#pragma unroll
-          for (int c = 0; c < 128; c += 8) {
-            a0 = max3(a0, __uint_as_float(s[c]), __uint_as_float(s[c + 1]));
-            a1 = max3(a1, __uint_as_float(s[c + 2]), __uint_as_float(s[c + 3]));
-            a2 = max3(a2, __uint_as_float(s[c + 4]), __uint_as_float(s[c + 5]));
-            a3 = max3(a3, __uint_as_float(s[c + 6]), __uint_as_float(s[c + 7]));
-          }
-          mx = fmaxf(fmaxf(a0, a1), fmaxf(a2, a3));
-          redo = __any_sync(0xffffffffu, mx * g.scale_log2 > m_ref + kRescaleThreshold);
-          if (!redo) sum = exp_pass(m_ref == neg_inf ? 0.f : m_ref, mx, true);
-#endif
-        }
-        if (redo) {
-          const float ms = mx * g.scale_log2;
-          float alpha = 1.f;
-          if (ms > m_ref + kRescaleThreshold) {   // also true when m_ref == -inf
-            alpha = fast_exp2(m_ref - ms);        // 0 when m_ref == -inf
-            m_ref = ms;
-          }
-          l *= alpha;
-#pragma unroll
-          for (int c4 = 0; c4 < 4; ++c4) {
-            uint32_t o[32];
-            tc_ld32(tO + c4 * 32, o);
-            tc_wait_ld();
-#pragma unroll
-            for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
-            tc_st32(tO + c4 * 32, o);
-          }
-          sum = exp_pass(m_ref == neg_inf ? 0.f : m_ref, mx, !PSA_OPTIMISTIC);
-        }
-#if PSA_SPLIT_P && PSA_OPTIMISTIC
-        if (j > 0) {  // the optimistic pass may not publish a half before it is confirmed
-          tc_wait_st();
-          tc_fence_before();
-          mbar_arrive(bar(kBarPHalf + qi));
-        }
-#endif
-        l += sum;
-        tc_wait_st();
-        tc_fence_before();
-        mbar_arrive(bar(kBarPReady + qi));
+        const uint32_t bh = bar(kBarPHalf + qi), br = bar(kBarPReady + qi);
+        if (nk == 128) softmax_slab<128>(tS, tO, m, j == 0, g.scale_log2, m_ref, l, bh, br);
+        else if (nk == 112) softmax_slab<112>(tS, tO, m, j == 0, g.scale_log2, m_ref, l, bh, br);
+        else if (nk == 96) softmax_slab<96>(tS, tO, m, j == 0, g.scale_log2, m_ref, l, bh, br);
+        else softmax_slab<64>(tS, tO, m, j == 0, g.scale_log2, m_ref, l, bh, br);
       }
       if (!ok) break;
       // ---- epilogue: out = O / l, lse = ln2 * (m_ref + log2 l)
@@ -882,12 +908,13 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       }
       tc_fence_before();
       mbar_arrive(bar(kBarOEmpty + qi));
-      int t0, h0, w0;
+      int t0, h0, w0, et, eh, ew, ntok, last;
       slab_origin(g, qb, sub0 + qi, t0, h0, w0);
+      slab_shape(g, sub0 + qi, et, eh, ew, ntok, last);
       {
-        const int wi_ = row % g.cw, hi_ = (row / g.cw) % g.ch, ti_ = row / (g.cw * g.ch);
+        const int wi_ = row % ew, hi_ = (row / ew) % eh, ti_ = row / (ew * eh);
         const int t = t0 + ti_, hh = h0 + hi_, ww = w0 + wi_;
-        if (t < g.T && hh < g.H && ww < g.W) {
+        if (row < ntok && t < g.T && hh < g.H && ww < g.W) {
           const long long tok = ((long long)t * g.H + hh) * g.W + ww;
           prm.lse[(long long)head * g.L + tok] = empty ? neg_inf : (m_ref + log2f(l)) * 0.6931471805599453f;
         }
@@ -896,8 +923,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       named_bar_sync(1 + qi, 128);
       if ((warp & 3) == 0 && lane == 0) {
         const uint32_t src = sbase + kOffQ + (uint32_t)qi * kSlabBytes;
-        tma_store_5d(&tm_o, src, 0, w0, h0, t0, head);
-        tma_store_5d(&tm_o, src + kHalfBytes, 64, w0, h0, t0, head);
+        tma_store_5d(&tms.o[last], src, 0, w0, h0, t0, head);
+        tma_store_5d(&tms.o[last], src + kHalfBytes, 64, w0, h0, t0, head);
         tma_store_commit();
         tma_store_wait_read();
         mbar_arrive(bar(kBarQEmpty + qi));
@@ -955,9 +982,8 @@ cudaError_t launch_plan(const HeadParamsArray& hp, const Geom& g, int head0, int
   return cudaGetLastError();
 }
 
-cudaError_t launch_attn(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to,
-                        const Geom& g, const WorkItem* items, const psa_head_params* hp_dev, int* ws_header,
-                        float* lse, int n_items, int n_sms, cudaStream_t stream) {
+cudaError_t launch_attn(const TensorMaps& tm, const Geom& g, const WorkItem* items, const psa_head_params* hp_dev,
+                        int* ws_header, float* lse, int n_items, int n_sms, cudaStream_t stream) {
   {  // per device, cheap: set on every call
     cudaError_t e = cudaFuncSetAttribute(attn_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemAlloc);
     if (e != cudaSuccess) return e;
@@ -971,7 +997,7 @@ cudaError_t launch_attn(const CUtensorMap& tq, const CUtensorMap& tk, const CUte
   prm.n_items = n_items;
   const int grid = n_items < n_sms ? n_items : n_sms;
   if (grid <= 0) return cudaSuccess;
-  attn_fwd_kernel<<<grid, kThreads, kSmemAlloc, stream>>>(tq, tk, tv, to, prm);
+  attn_fwd_kernel<<<grid, kThreads, kSmemAlloc, stream>>>(tm, prm);
   return cudaGetLastError();
 }
 

@@ -21,6 +21,8 @@ struct Geom {
   int ct, ch, cw;          // 128-token slab = one TMA box (ct*ch*cw == 128)
   int n_sub;               // slabs per mask block (1..3)
   int sub_axis;            // axis along which the slabs of a block stack: 0 = t, 1 = h, 2 = w
+  int c_last;              // extent of a block's LAST slab along sub_axis (<= the full slab's)
+  int n_last;              // tokens of that last slab: 128, 112, 96 or 64
   int n_heads;
   int items_per_block;     // work items per query block = ceil(n_sub / 2)
   float scale_log2;        // softmax scale times log2(e)

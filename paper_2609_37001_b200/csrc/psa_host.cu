@@ -17,9 +17,11 @@ cudaError_t launch_mask_build(const HeadParamsArray& hp, const int* head_bases, 
                               int n_sms, cudaStream_t stream, int* launches);
 cudaError_t launch_plan(const HeadParamsArray& hp, const Geom& g, int head0, int n_heads_here, int* ws_header,
                         psa_head_params* hp_dev, WorkItem* items, cudaStream_t stream);
-cudaError_t launch_attn(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to,
-                        const Geom& g, const WorkItem* items, const psa_head_params* hp_dev, int* ws_header,
-                        float* lse, int n_items, int n_sms, cudaStream_t stream);
+struct TensorMaps {
+  CUtensorMap q[2], k[2], v[2], o[2];  // [0]: full 128-token slab box, [1]: a block's last slab
+};
+cudaError_t launch_attn(const TensorMaps& tm, const Geom& g, const WorkItem* items, const psa_head_params* hp_dev,
+                        int* ws_header, float* lse, int n_items, int n_sms, cudaStream_t stream);
 cudaError_t launch_wait_probe(int* ws_header, unsigned long long limit_ns, cudaStream_t stream);
 }  // namespace psa
 
@@ -86,22 +88,30 @@ int make_geom(const psa_problem* prob, int T, int H, int W, bool for_attn, Geom*
   g->sub_axis = 0;
   g->items_per_block = 1;
   if (for_attn) {
+    g->c_last = 1;
+    g->n_last = kSlabTokens;
     if (prob->head_dim != kHeadDim) return PSA_ERR_UNSUPPORTED;
     if (!(prob->scale > 0.f) || !std::isfinite(prob->scale)) return PSA_ERR_INVALID_ARG;
+    // Split the block into slabs along its outermost axis of extent > 1: full slabs of 128
+    // tokens, and a last slab that may be shorter (112, 96 or 64 tokens) so that blocks such
+    // as 1x15x16 tile a 45-row grid without padding.
     const long long tokens = (long long)t.bt * t.bh * t.bw;
-    if (tokens != 128 && tokens != 256 && tokens != 384) return PSA_ERR_UNSUPPORTED;
-    const int n_sub = (int)(tokens / kSlabTokens);
-    // split the block into n_sub slabs along its outermost axis of extent > 1
-    if (t.bt > 1 || (t.bh == 1 && t.bw == 1)) {
-      if (t.bt % n_sub) return PSA_ERR_UNSUPPORTED;
-      g->ct = t.bt / n_sub; g->sub_axis = 0;
-    } else if (t.bh > 1) {
-      if (t.bh % n_sub) return PSA_ERR_UNSUPPORTED;
-      g->ch = t.bh / n_sub; g->sub_axis = 1;
-    } else {
-      if (t.bw % n_sub) return PSA_ERR_UNSUPPORTED;
-      g->cw = t.bw / n_sub; g->sub_axis = 2;
-    }
+    if (tokens < 128 || tokens > 384) return PSA_ERR_UNSUPPORTED;
+    int axis, extent;
+    long long other;
+    if (t.bt > 1 || (t.bh == 1 && t.bw == 1)) { axis = 0; extent = t.bt; other = (long long)t.bh * t.bw; }
+    else if (t.bh > 1) { axis = 1; extent = t.bh; other = (long long)t.bt * t.bw; }
+    else { axis = 2; extent = t.bw; other = (long long)t.bt * t.bh; }
+    if (other > kSlabTokens || (kSlabTokens % other) != 0) return PSA_ERR_UNSUPPORTED;
+    const int c0 = (int)(kSlabTokens / other);
+    const int n_sub = (extent + c0 - 1) / c0;
+    const int c_last = extent - (n_sub - 1) * c0;
+    const int n_last = (int)(c_last * other);
+    if (n_sub > 3 || !(n_last == 128 || n_last == 112 || n_last == 96 || n_last == 64)) return PSA_ERR_UNSUPPORTED;
+    if (axis == 0) g->ct = c0; else if (axis == 1) g->ch = c0; else g->cw = c0;
+    g->sub_axis = axis;
+    g->c_last = c_last;
+    g->n_last = n_last;
     if (g->ct > 128 || g->ch > 128 || g->cw > 128) return PSA_ERR_UNSUPPORTED;
     if (g->Tp > kMaxTp || g->Sp > kMaxSp) return PSA_ERR_UNSUPPORTED;
     g->n_sub = n_sub;
@@ -150,18 +160,34 @@ int ensure_workspace(Workspace* w, size_t bytes) {
   return PSA_OK;
 }
 
-int encode_map(CUtensorMap* tm, const void* base, const Geom& g, const psa_problem* prob, int n_heads_here) {
+// `last`: box of a block's last (possibly shorter) slab instead of the full 128-token slab.
+int encode_map(CUtensorMap* tm, const void* base, const Geom& g, const psa_problem* prob, int n_heads_here,
+               bool last = false) {
   const cuuint64_t dims[5] = {(cuuint64_t)kHeadDim, (cuuint64_t)g.W, (cuuint64_t)g.H, (cuuint64_t)g.T,
                               (cuuint64_t)n_heads_here};
   const cuuint64_t st = (cuuint64_t)prob->stride_token * 2;
   const cuuint64_t strides[4] = {st, st * g.W, st * g.W * g.H,
                                  n_heads_here > 1 ? (cuuint64_t)prob->stride_head * 2 : st * g.W * g.H * g.T};
-  const cuuint32_t box[5] = {64, (cuuint32_t)g.cw, (cuuint32_t)g.ch, (cuuint32_t)g.ct, 1};
+  cuuint32_t box[5] = {64, (cuuint32_t)g.cw, (cuuint32_t)g.ch, (cuuint32_t)g.ct, 1};
+  if (last) box[3 - g.sub_axis] = (cuuint32_t)g.c_last;
   const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
   const CUresult r = g_encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(base), dims, strides, box,
                               estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? PSA_OK : PSA_ERR_INVALID_ARG;
+}
+
+// The four tensors, each with the full-slab box ([0]) and the last-slab box ([1]).
+int encode_maps(TensorMaps* tm, const void* q, const void* k, const void* v, void* out, const Geom& g,
+                const psa_problem* prob, int n_heads_here) {
+  int rc;
+  for (int last = 0; last < 2; ++last) {
+    if ((rc = encode_map(&tm->q[last], q, g, prob, n_heads_here, last != 0)) != PSA_OK) return rc;
+    if ((rc = encode_map(&tm->k[last], k, g, prob, n_heads_here, last != 0)) != PSA_OK) return rc;
+    if ((rc = encode_map(&tm->v[last], v, g, prob, n_heads_here, last != 0)) != PSA_OK) return rc;
+    if ((rc = encode_map(&tm->o[last], out, g, prob, n_heads_here, last != 0)) != PSA_OK) return rc;
+  }
+  return PSA_OK;
 }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -316,18 +342,17 @@ int psa_attn_fwd(const void* q, const void* k, const void* v, void* out, float* 
     std::memset(&hp, 0, sizeof(hp));
     for (int h = 0; h < n_here; ++h) hp.p[h] = head_params[head0 + h];
     const long long eoff = (long long)head0 * prob->stride_head;
-    CUtensorMap tq, tk, tv, to;
-    if ((rc = encode_map(&tq, static_cast<const uint16_t*>(q) + eoff, g, prob, n_here)) != PSA_OK) return rc;
-    if ((rc = encode_map(&tk, static_cast<const uint16_t*>(k) + eoff, g, prob, n_here)) != PSA_OK) return rc;
-    if ((rc = encode_map(&tv, static_cast<const uint16_t*>(v) + eoff, g, prob, n_here)) != PSA_OK) return rc;
-    if ((rc = encode_map(&to, static_cast<uint16_t*>(out) + eoff, g, prob, n_here)) != PSA_OK) return rc;
+    TensorMaps tm;
+    if ((rc = encode_maps(&tm, static_cast<const uint16_t*>(q) + eoff, static_cast<const uint16_t*>(k) + eoff,
+                          static_cast<const uint16_t*>(v) + eoff, static_cast<uint16_t*>(out) + eoff, g, prob, n_here)) != PSA_OK)
+      return rc;
     Geom gh = g;
     gh.n_heads = n_here;
     if (launch_plan(hp, gh, 0, n_here, ws_header, hp_dev, items, st) != cudaSuccess) return PSA_ERR_CUDA;
     ++g_launches;
     const int n_items = n_here * g.NB * g.items_per_block;
     if (g_ev_start && g_ev_stop) cudaEventRecord(g_ev_start, st);
-    if (launch_attn(tq, tk, tv, to, gh, items, hp_dev, ws_header, lse + (long long)head0 * g.L, n_items, ws->n_sms, st) !=
+    if (launch_attn(tm, gh, items, hp_dev, ws_header, lse + (long long)head0 * g.L, n_items, ws->n_sms, st) !=
         cudaSuccess)
       return PSA_ERR_CUDA;
     if (g_ev_start && g_ev_stop) cudaEventRecord(g_ev_stop, st);
@@ -373,16 +398,13 @@ int psa_attn_fwd_noalloc(const void* q, const void* k, const void* v, void* out,
   HeadParamsArray hp;
   std::memset(&hp, 0, sizeof(hp));
   for (int h = 0; h < prob->n_heads; ++h) hp.p[h] = head_params[h];
-  CUtensorMap tq, tk, tv, to;
-  if ((rc = encode_map(&tq, q, g, prob, prob->n_heads)) != PSA_OK) return rc;
-  if ((rc = encode_map(&tk, k, g, prob, prob->n_heads)) != PSA_OK) return rc;
-  if ((rc = encode_map(&tv, v, g, prob, prob->n_heads)) != PSA_OK) return rc;
-  if ((rc = encode_map(&to, out, g, prob, prob->n_heads)) != PSA_OK) return rc;
+  TensorMaps tm;
+  if ((rc = encode_maps(&tm, q, k, v, out, g, prob, prob->n_heads)) != PSA_OK) return rc;
   // The planning kernel clears the header words (status, ticket) and rewrites the parameter
   // records and every work item of this call, so nothing of the previous call is read.
   if (launch_plan(hp, g, 0, prob->n_heads, header, hp_dev, items, st) != cudaSuccess) return PSA_ERR_CUDA;
   ++g_launches;
-  if (launch_attn(tq, tk, tv, to, g, items, hp_dev, header, lse, (int)n_items_ll, ws->n_sms, st) != cudaSuccess)
+  if (launch_attn(tm, g, items, hp_dev, header, lse, (int)n_items_ll, ws->n_sms, st) != cudaSuccess)
     return PSA_ERR_CUDA;
   ++g_launches;
   if (status_detail) {

@@ -100,6 +100,9 @@ def test_tiny_every_row(B, name):
     ((5, 9, 40), (1, 4, 32), [(2, 1, 3, 2, 0, 3), (5, 0, INF, 1, 0, 1)]),         # 128-token blocks, ragged h, w
     ((2, 30, 10), (2, 32, 4), [(1, 0, INF, 2, -1, INF), (1, 0, 1, 1, 1, 2)]),     # slab stacks along t
     ((1, 4, 100), (1, 1, 256), [(1, 0, INF, 1, 0, INF)]),                         # slab stacks along w
+    ((3, 45, 32), (1, 15, 16), [(2, 0, INF, 2, 0, 3), (1, 1, 2, 6, 0, INF)]),      # 240-token blocks: 128 + 112 slabs
+    ((2, 30, 40), (1, 12, 16), [(2, 0, 2, 2, 0, 3), (1, 0, INF, 9, 0, INF)]),      # 192 = 128 + 64, ragged h and w
+    ((2, 28, 16), (1, 14, 16), [(1, 0, INF, 1, 1, INF)]),                          # 224 = 128 + 96
     ((4, 16, 16), (1, 16, 16), [(1, 7, INF, 1, 0, INF)]),                         # offset beyond the grid: all rows empty
 ])
 def test_small_shapes_every_row(B, grid, tile, params):
@@ -149,6 +152,7 @@ def _sampled_rows(grid, tile, seed):
 @pytest.mark.parametrize("name,heads", [
     ("wan13b_480p", None),
     ("wan14b_720p", list(range(0, 40, 5))),
+    ("wan14b_720p_b1x16x16", [2, 17, 31]),
     ("wan14b_720p_b3x8x16", [0, 13, 26]),
     ("hunyuan_720p", [1, 8, 15, 22]),
     ("sweep_00", [0]), ("sweep_25", [3]), ("sweep_50", [5]), ("sweep_75", [7]), ("sweep_90", [39]),
