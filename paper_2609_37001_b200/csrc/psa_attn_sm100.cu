@@ -235,6 +235,9 @@ __device__ __forceinline__ void exp2_poly_pair(uint64_t x2, float& p0, float& p1
 #ifndef PSA_EMU_PAIRS
 #define PSA_EMU_PAIRS 0   // of every 4 pairs of probabilities, this many use exp2_poly_pair (0: all ex2.approx)
 #endif
+#ifndef PSA_MAX8
+#define PSA_MAX8 1        // eight row-max chains instead of four
+#endif
 #ifndef PSA_SPLIT_P
 #define PSA_SPLIT_P 1     // publish P in two halves of 64 keys
 #endif
@@ -268,6 +271,20 @@ __device__ __forceinline__ bool elect_one() {
   asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(pred));
   return pred != 0;
 }
+
+// Developer knob (-DPSA_TRACE): CTA 0 records cycle stamps of its second work item.
+#ifdef PSA_TRACE
+__device__ long long g_trace[4 * 64 * 8];
+__device__ long long g_trace_items[2 * 256 * 4];
+#define TRACE(role, j, k)                                                                     \
+  do {                                                                                          \
+    if (blockIdx.x == 0 && n == 1 && (j) < 64 && (threadIdx.x & 31) == 0 &&                     \
+        ((threadIdx.x >> 5) & 3) == ((role) < 2 ? 0 : 1))                                       \
+      g_trace[((role) * 64 + (j)) * 8 + (k)] = clock64();                                       \
+  } while (0)
+#else
+#define TRACE(role, j, k) do { } while (0)
+#endif
 
 // ----------------------------------------------------------------------------- planning
 // Work order: per head, query blocks ranked by attended key-block count (largest first),
@@ -361,14 +378,19 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t lo) { return ((uint64_t)k
 // Online-softmax step of one query row (one thread) for one key slab of NK keys.
 //   tS: TMEM address of the row's scores (fp32, NK columns); the bf16 probabilities are written
 //       back over the first NK/2 columns.  tO: the row's output accumulator (128 fp32 columns).
-//   meta: [0] != 0 marks a slab with padded key positions, [1..4] = validity bits of its keys.
+//   meta: validity bits of the slab's keys (bit c of word c/32); all ones when nothing is padded.
 //   m_ref / l: running reference maximum (scaled log2 domain) and running sum.
 // The reference maximum is lazy: it moves only when the slab's maximum exceeds it by more than
 // kRescaleThreshold, so exponentials stay below 2^threshold and O is rarely rescaled.
 template <int NK>
-__device__ __forceinline__ void softmax_slab(uint32_t tS, uint32_t tO, const uint32_t* meta, bool first,
+__device__ __forceinline__ void softmax_slab(uint32_t tS, uint32_t tO, const uint4 meta, bool first,
                                              float scale_log2, float& m_ref, float& l, uint32_t bar_half,
-                                             uint32_t bar_ready) {
+                                             uint32_t bar_ready, long long* tr = nullptr) {
+#ifdef PSA_TRACE
+#define STAMP(k) do { if (tr) tr[k] = clock64(); } while (0)
+#else
+#define STAMP(k) do { } while (0)
+#endif
   constexpr int NFULL = NK / 32, REM = NK % 32;
   static_assert(NK % 16 == 0 && NK >= 64 && NK <= 128 && (REM == 0 || REM == 16), "unsupported slab width");
   const float neg_inf = __int_as_float(0xff800000);
@@ -377,12 +399,26 @@ __device__ __forceinline__ void softmax_slab(uint32_t tS, uint32_t tO, const uin
   for (int c4 = 0; c4 < NFULL; ++c4) tc_ld32(tS + c4 * 32, s + c4 * 32);
   if (REM) tc_ld16(tS + NFULL * 32, s + NFULL * 32);
   tc_wait_ld();
-  if (meta[0] != 0u) {  // 3D-padding: padded key positions score -inf
-    const uint32_t v[4] = {meta[1], meta[2], meta[3], meta[4]};
+  STAMP(1);
+  if ((meta.x & meta.y & meta.z & meta.w) != 0xffffffffu) {  // 3D-padding: padded key positions score -inf
+    const uint32_t v[4] = {meta.x, meta.y, meta.z, meta.w};
 #pragma unroll
     for (int c = 0; c < NK; ++c)
       if (!((v[c >> 5] >> (c & 31)) & 1u)) s[c] = 0xff800000u;
   }
+  STAMP(7);
+#if PSA_MAX8
+  // eight independent chains (NK is a multiple of 16): shorter dependency depth
+  float a[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) a[i] = fmaxf(__uint_as_float(s[2 * i]), __uint_as_float(s[2 * i + 1]));
+#pragma unroll
+  for (int c = 16; c < NK; c += 16) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) a[i] = max3(a[i], __uint_as_float(s[c + 2 * i]), __uint_as_float(s[c + 2 * i + 1]));
+  }
+  const float ms = fmaxf(fmaxf(max3(a[0], a[1], a[2]), max3(a[3], a[4], a[5])), fmaxf(a[6], a[7])) * scale_log2;
+#else
   float a0 = neg_inf, a1 = neg_inf, a2 = neg_inf, a3 = neg_inf;
 #pragma unroll
   for (int c = 0; c < NK; c += 8) {
@@ -392,6 +428,8 @@ __device__ __forceinline__ void softmax_slab(uint32_t tS, uint32_t tO, const uin
     a3 = max3(a3, __uint_as_float(s[c + 6]), __uint_as_float(s[c + 7]));
   }
   const float ms = fmaxf(fmaxf(a0, a1), fmaxf(a2, a3)) * scale_log2;
+#endif
+  STAMP(5);   // (overwritten later by the half-way stamp when tracing the split; read before)
   if (first) {
     m_ref = ms;  // first slab of the item: nothing accumulated yet
   } else {
@@ -415,6 +453,7 @@ __device__ __forceinline__ void softmax_slab(uint32_t tS, uint32_t tO, const uin
     }
   }
   const float m_use = (m_ref == neg_inf) ? 0.f : m_ref;
+  STAMP(2);
   const uint64_t sc2 = pack2(scale_log2, scale_log2), negm2 = pack2(-m_use, -m_use);
   uint64_t sum2 = pack2(0.f, 0.f);
   // probabilities exp2(scale*s - m_use), bf16, written over the scores in chunks of 32 keys
@@ -443,9 +482,11 @@ __device__ __forceinline__ void softmax_slab(uint32_t tS, uint32_t tO, const uin
     tc_st16(tS + c4 * 16, pk);
 #if PSA_SPLIT_P
     if (c4 == 1) {  // the first 64 keys are final: their P V MMAs may start
+      STAMP(5);
       tc_wait_st();
       tc_fence_before();
       mbar_arrive(bar_half);
+      STAMP(3);
     }
 #endif
   }
@@ -457,9 +498,11 @@ __device__ __forceinline__ void softmax_slab(uint32_t tS, uint32_t tO, const uin
   float sum0, sum1;
   unpack2(sum2, sum0, sum1);
   l += sum0 + sum1;
+  STAMP(6);
   tc_wait_st();
   tc_fence_before();
   mbar_arrive(bar_ready);
+#undef STAMP
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -638,8 +681,7 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
                 if (!ok) break;
                 if (lane == 0) {
                   uint32_t* m = meta + (kv_g % kMetaRing) * 8;
-                  m[0] = edge ? 1u : 0u;
-                  m[1] = vw0; m[2] = vw1; m[3] = vw2; m[4] = vw3;
+                  m[0] = vw0; m[1] = vw1; m[2] = vw2; m[3] = vw3;
                   const uint32_t pb = bar(kBarPairFull + pair_g % kNumPairBars);
                   mbar_expect_tx(pb, (uint32_t)((have_prev ? pntok : 0) + ntok) * 256u);
                   if (have_prev) {
@@ -743,6 +785,12 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
       if (!next_item(n, wi)) break;
       const int nq = wi.w >> 16;
       const int n_kv = wi.z * g.n_sub;
+#ifdef PSA_TRACE
+      if ((blockIdx.x == 0 || blockIdx.x == 77) && n < 256 && lane == 0) {
+        long long* r = g_trace_items + ((blockIdx.x == 0 ? 0 : 1) * 256 + n) * 4;
+        r[0] = clock64(); r[1] = n_kv; r[2] = wi.x; r[3] = (long long)globaltimer_ns();
+      }
+#endif
 #pragma unroll
       for (int i = 0; i < 2; ++i) {
         if (i >= nq) break;
@@ -781,8 +829,10 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
           sub = (sub + 1 == g.n_sub) ? 0 : sub + 1;
           const int nk_next = (sub == g.n_sub - 1) ? g.n_last : kSlabTokens;
           // V_j and (unless this is the last slab) K_{j+1} arrive under one barrier
+          TRACE(2, j, 5);
           ok = mbar_wait_warp(bar(kBarPairFull + pair_g % kNumPairBars), (pair_g / kNumPairBars) & 1u, abort_flag, 0x211);
           if (!ok) break;
+          TRACE(2, j, 3);
           ++pair_g;
           const bool more = (j + 1 < n_kv);
           const uint32_t vslot = tile_g % kNumSlots;
@@ -796,12 +846,14 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
             ok = mbar_wait_warp(bar(kBarPHalf + i), cs & 1u, abort_flag, 0x224 + i);
             if (!ok) break;
             tc_fence_after();
+            TRACE(2 + i, j, 0);
             if (elect_one()) issue_pv_half(i, vslot, 0, j > 0, nk_cur);
 #endif
             ok = mbar_wait_warp(bar(kBarPReady + i), cs & 1u, abort_flag, 0x220 + i);
             if (!ok) break;
             if (i == 0) ++cnt_s0; else ++cnt_s1;
             tc_fence_after();
+            TRACE(2 + i, j, 1);
             if (elect_one()) {
 #if PSA_SPLIT_P
               issue_pv_half(i, vslot, 1, true, nk_cur);
@@ -819,6 +871,7 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
               }
             }
             __syncwarp();
+            TRACE(2 + i, j, 2);
           }
         }
         if (!ok) break;
@@ -864,12 +917,21 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
         if (!ok) break;
         ++cnt_s;
         tc_fence_after();
-        const uint32_t* m = meta + (kv_g % kMetaRing) * 8;
+        TRACE(qi, j, 0);
+        // Read the slab's validity words first: shared memory is busy feeding the tensor core,
+        // so the load's latency is overlapped with the TMEM loads that follow.
+        const uint4 m = *reinterpret_cast<const uint4*>(meta + (kv_g % kMetaRing) * 8);
         const uint32_t bh = bar(kBarPHalf + qi), br = bar(kBarPReady + qi);
-        if (nk == 128) softmax_slab<128>(tS, tO, m, j == 0, g.scale_log2, m_ref, l, bh, br);
-        else if (nk == 112) softmax_slab<112>(tS, tO, m, j == 0, g.scale_log2, m_ref, l, bh, br);
-        else if (nk == 96) softmax_slab<96>(tS, tO, m, j == 0, g.scale_log2, m_ref, l, bh, br);
-        else softmax_slab<64>(tS, tO, m, j == 0, g.scale_log2, m_ref, l, bh, br);
+#ifdef PSA_TRACE
+        long long* tr = (blockIdx.x == 0 && n == 1 && j < 64 && (threadIdx.x & 127) == 0) ? g_trace + (qi * 64 + j) * 8 : nullptr;
+#else
+        long long* tr = nullptr;
+#endif
+        if (nk == 128) softmax_slab<128>(tS, tO, m, j == 0, g.scale_log2, m_ref, l, bh, br, tr);
+        else if (nk == 112) softmax_slab<112>(tS, tO, m, j == 0, g.scale_log2, m_ref, l, bh, br, tr);
+        else if (nk == 96) softmax_slab<96>(tS, tO, m, j == 0, g.scale_log2, m_ref, l, bh, br, tr);
+        else softmax_slab<64>(tS, tO, m, j == 0, g.scale_log2, m_ref, l, bh, br, tr);
+        TRACE(qi, j, 4);
       }
       if (!ok) break;
       // ---- epilogue: out = O / l, lse = ln2 * (m_ref + log2 l)
@@ -1003,3 +1065,12 @@ cudaError_t launch_attn(const TensorMaps& tm, const Geom& g, const WorkItem* ite
 
 }  // namespace psa
 
+
+#ifdef PSA_TRACE
+extern "C" int psa_debug_read_trace(long long* out, int n) {
+  return (int)cudaMemcpyFromSymbol(out, psa::g_trace, sizeof(long long) * n);
+}
+extern "C" int psa_debug_read_items(long long* out, int n) {
+  return (int)cudaMemcpyFromSymbol(out, psa::g_trace_items, sizeof(long long) * n);
+}
+#endif
