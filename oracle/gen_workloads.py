@@ -120,6 +120,18 @@ def main():
     wl.append(describe("ragged_75", grid, tile, [closest(c, 0.75)] * 40, "ragged grid, ~75% sparsity", 0x50534105))
     Tp, Hp, Wp = O.block_grid(*grid, tile)
     wl.append(describe("ragged_dense", grid, tile, [[Tp, 0, INF, Hp * Wp, 0, INF]] * 40, "ragged grid, all-covering", 0x50534105))
+    # N1. HunyuanVideo 768x1280 (30x48x80, Table 2 / Table 3b): no padding with 1x16x16 or with the paper's
+    #     6x8x8 block; plus the 60/70/80/90 % levels of Table 3b (all heads share one parameter set per level)
+    grid = (30, 48, 80)
+    for name, tile in (("hunyuan_768p", (1, 16, 16)), ("hunyuan_768p_b6x8x8", (6, 8, 8))):
+        rng = np.random.Generator(np.random.Philox(key=0x50534106))
+        wl.append(describe(name, grid, tile, draw_heads(rng, candidates(*grid, tile), 24, 0.50, 0.85),
+                           "24 heads, 50-85% tile sparsity, temporal/spatial/joint in turn", 0x50534106))
+    tile = (1, 16, 16)
+    c = candidates(*grid, tile)
+    for level in (60, 70, 80, 90):
+        wl.append(describe(f"hy768_sweep_{level}", grid, tile, [closest(c, level / 100.0)] * 24,
+                           f"HunyuanVideo 768p sparsity sweep, target {level}%", 0x50534106))
     with open(OUT, "w") as f:
         json.dump({"_generator": "oracle/gen_workloads.py", "inf_stride": INF, "workloads": wl}, f, indent=1)
     for w in wl:

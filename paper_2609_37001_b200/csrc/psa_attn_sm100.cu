@@ -45,8 +45,10 @@ constexpr uint32_t kOffMaskT = kOffMeta + kMetaRing * 32;       // kMaxTp / 32 w
 constexpr uint32_t kOffMaskS = kOffMaskT + (kMaxTp / 32) * 4;   // kMaxSp / 32 words
 constexpr uint32_t kOffSched = kOffMaskS + (kMaxSp / 32) * 4;   // two published work items
 constexpr uint32_t kOffMisc = kOffSched + 32;                   // tmem base, abort flag
-constexpr uint32_t kSmemBytes = kOffMisc + 16;
+constexpr uint32_t kOffXchg = kOffMisc + 16;                    // split-KV merge: (m, l) of 128 rows
+constexpr uint32_t kSmemBytes = kOffXchg + 128 * 8;
 constexpr uint32_t kSmemAlloc = kSmemBytes + 1024;              // slack for manual alignment
+static_assert(kSmemAlloc <= 232448, "exceeds the 227 KB of shared memory a CTA may use");
 
 // ----------------------------------------------------------------------------- PTX
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -326,7 +328,9 @@ plan_kernel(const HeadParamsArray hp, const Geom g, int head0, int* __restrict__
     for (int it = 0; it < ipb; ++it) {
       const int sub0 = 2 * it;
       const int nq = (g.n_sub - sub0) >= 2 ? 2 : 1;
-      out[(size_t)it * g.NB + pos] = make_int4(h, qb, c, sub0 | (nq << 16));
+      // A single-slab item runs in split-KV mode: both softmax warpgroups work on that one
+      // query slab, one on the even and one on the odd key slabs (flag in bit 24).
+      out[(size_t)it * g.NB + pos] = make_int4(h, qb, c, sub0 | (nq << 16) | ((nq == 1 ? 1 : 0) << 24));
     }
   }
 }
@@ -602,7 +606,8 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
       wi.y = __shfl_sync(0xffffffffu, wi.y, 0);
       wi.w = __shfl_sync(0xffffffffu, wi.w, 0);
       if (wi.x < 0) break;
-      const int head = wi.x, qb = wi.y, sub0 = wi.w & 0xffff, nq = wi.w >> 16;
+      const int head = wi.x, qb = wi.y, sub0 = wi.w & 0xffff, nq = (wi.w >> 16) & 0xff;
+      const int lag = (wi.w >> 24) ? 2 : 1;   // V_j travels with K_{j+lag} (2 in split-KV mode)
       const psa_head_params p = prm.hp_dev[head];
       const int tq = qb / g.Sp, sq = qb % g.Sp;
       // attended key-block coordinates of this query block, one bit per block coordinate
@@ -636,10 +641,10 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
         if (i == 0) ++it_q0; else ++it_q1;
       }
       if (!ok) break;
-      // key / value slabs in ascending key-block id
-      bool have_prev = false;
-      int pt0 = 0, ph0 = 0, pw0 = 0;  // origin of the previous slab (its V is still to be loaded)
-      int plast = 0, pntok = kSlabTokens;
+      // key / value slabs in ascending key-block id.  Up to `lag` slabs wait for their V load.
+      int npend = 0;
+      int at0 = 0, ah0 = 0, aw0 = 0, alast = 0, antok = kSlabTokens;  // oldest pending slab
+      int bt0 = 0, bh0 = 0, bw0 = 0, blast = 0, bntok = kSlabTokens;  // newer pending slab (lag 2)
       for (int tw = 0; ok && tw < g.Tp; tw += 32) {
         uint32_t mt = maskT[tw >> 5];
         while (ok && mt) {
@@ -669,11 +674,12 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
                   c += 32;
                   vw3 = __ballot_sync(0xffffffffu, (t0 + c / ehw < g.T) && (h0 + (c / ew) % eh < g.H) && (w0 + c % ew < g.W));
                 }
-                // slots: [V of the previous slab,] K of this slab
+                // slots: [V of the oldest pending slab,] K of this slab
+                const bool with_v = (npend == lag);
                 const uint32_t v_slot = tile_g % kNumSlots, v_use = tile_g / kNumSlots;
-                const uint32_t k_tile = tile_g + (have_prev ? 1u : 0u);
+                const uint32_t k_tile = tile_g + (with_v ? 1u : 0u);
                 const uint32_t k_slot = k_tile % kNumSlots, k_use = k_tile / kNumSlots;
-                if (have_prev) {
+                if (with_v) {
                   ok = mbar_wait_warp(bar(kBarSlotEmpty + v_slot), (v_use & 1u) ^ 1u, abort_flag, 0x111);
                   if (!ok) break;
                 }
@@ -683,42 +689,49 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
                   uint32_t* m = meta + (kv_g % kMetaRing) * 8;
                   m[0] = vw0; m[1] = vw1; m[2] = vw2; m[3] = vw3;
                   const uint32_t pb = bar(kBarPairFull + pair_g % kNumPairBars);
-                  mbar_expect_tx(pb, (uint32_t)((have_prev ? pntok : 0) + ntok) * 256u);
-                  if (have_prev) {
+                  mbar_expect_tx(pb, (uint32_t)((with_v ? antok : 0) + ntok) * 256u);
+                  if (with_v) {
                     const uint32_t dv = sbase + kOffRing + v_slot * kSlabBytes;
-                    tma_load_5d(dv, &tms.v[plast], pb, 0, pw0, ph0, pt0, head);
-                    tma_load_5d(dv + kHalfBytes, &tms.v[plast], pb, 64, pw0, ph0, pt0, head);
+                    tma_load_5d(dv, &tms.v[alast], pb, 0, aw0, ah0, at0, head);
+                    tma_load_5d(dv + kHalfBytes, &tms.v[alast], pb, 64, aw0, ah0, at0, head);
                   }
                   const uint32_t dk = sbase + kOffRing + k_slot * kSlabBytes;
                   tma_load_5d(dk, &tms.k[last], pb, 0, w0, h0, t0, head);
                   tma_load_5d(dk + kHalfBytes, &tms.k[last], pb, 64, w0, h0, t0, head);
                 }
-                plast = last;
-                pntok = ntok;
                 tile_g = k_tile + 1;
                 ++pair_g;
                 ++kv_g;
-                have_prev = true;
-                pt0 = t0; ph0 = h0; pw0 = w0;
+                // queue this slab's V
+                if (with_v) {
+                  if (lag == 2) { at0 = bt0; ah0 = bh0; aw0 = bw0; alast = blast; antok = bntok; }
+                  --npend;
+                }
+                if (npend == 0) { at0 = t0; ah0 = h0; aw0 = w0; alast = last; antok = ntok; }
+                else { bt0 = t0; bh0 = h0; bw0 = w0; blast = last; bntok = ntok; }
+                ++npend;
               }
             }
           }
         }
       }
-      if (ok && have_prev) {  // V of the item's last slab
+      while (ok && npend > 0) {  // V of the item's last slab(s), one pair barrier each
         const uint32_t v_slot = tile_g % kNumSlots, v_use = tile_g / kNumSlots;
         ok = mbar_wait_warp(bar(kBarSlotEmpty + v_slot), (v_use & 1u) ^ 1u, abort_flag, 0x112);
         if (!ok) break;
         if (lane == 0) {
           const uint32_t pb = bar(kBarPairFull + pair_g % kNumPairBars);
-          mbar_expect_tx(pb, (uint32_t)pntok * 256u);
+          mbar_expect_tx(pb, (uint32_t)antok * 256u);
           const uint32_t dv = sbase + kOffRing + v_slot * kSlabBytes;
-          tma_load_5d(dv, &tms.v[plast], pb, 0, pw0, ph0, pt0, head);
-          tma_load_5d(dv + kHalfBytes, &tms.v[plast], pb, 64, pw0, ph0, pt0, head);
+          tma_load_5d(dv, &tms.v[alast], pb, 0, aw0, ah0, at0, head);
+          tma_load_5d(dv + kHalfBytes, &tms.v[alast], pb, 64, aw0, ah0, at0, head);
         }
         ++tile_g;
         ++pair_g;
+        at0 = bt0; ah0 = bh0; aw0 = bw0; alast = blast; antok = bntok;
+        --npend;
       }
+      if (!ok) break;
     }
     // Let every load that was issued land before the CTA retires: wait for the last armed
     // phase of each pair barrier and of the Q barriers (bounded; the abort flag no longer
@@ -756,13 +769,14 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
 
     // S_i = Q_i K^T over head_dim = 128: 8 MMAs of K = 16; both operands K-major, SW128.
     // nk = keys of the slab (N of the instruction): 128, or fewer for a block's last slab.
-    auto issue_qk = [&](int i, uint32_t kslot, int nk) {
-      const uint32_t a0 = q_lo + (uint32_t)i * kSlabStep, b0 = ring_lo_k + kslot * kSlabStep;
+    // iq: Q buffer; it: S tile written (they differ only in split-KV items).
+    auto issue_qk = [&](int iq, uint32_t kslot, int nk, int it) {
+      const uint32_t a0 = q_lo + (uint32_t)iq * kSlabStep, b0 = ring_lo_k + kslot * kSlabStep;
       const uint32_t idesc = instr_desc(false, (uint32_t)nk);
 #pragma unroll
       for (int kk = 0; kk < 8; ++kk) {
         const uint32_t off = (uint32_t)(kk >> 2) * (kHalfBytes >> 4) + (uint32_t)(kk & 3) * 2u;
-        tc_mma_ss(tmem + (uint32_t)i * 128u, make_desc(a0 + off), make_desc(b0 + off), idesc, kk > 0 ? 1u : 0u);
+        tc_mma_ss(tmem + (uint32_t)it * 128u, make_desc(a0 + off), make_desc(b0 + off), idesc, kk > 0 ? 1u : 0u);
       }
     };
     // O_i (+)= P_i V over 128 keys: 8 MMAs of K = 16; A = bf16 P in TMEM (8 columns per
@@ -780,10 +794,14 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
       }
     };
 
+    uint32_t it_o0 = 0, it_o1 = 0;    // items in which accumulator O_i was used
+    auto nk_of = [&](int j) -> int { return (j % g.n_sub == g.n_sub - 1) ? g.n_last : kSlabTokens; };
+
     for (uint32_t n = 0; ok; ++n) {
       WorkItem wi;
       if (!next_item(n, wi)) break;
-      const int nq = wi.w >> 16;
+      const int nq = (wi.w >> 16) & 0xff;
+      const bool split = (wi.w >> 24) != 0;
       const int n_kv = wi.z * g.n_sub;
 #ifdef PSA_TRACE
       if ((blockIdx.x == 0 || blockIdx.x == 77) && n < 256 && lane == 0) {
@@ -791,18 +809,82 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
         r[0] = clock64(); r[1] = n_kv; r[2] = wi.x; r[3] = (long long)globaltimer_ns();
       }
 #endif
+      // which accumulators this item uses: both for a two-slab item, and for a split-KV item
+      // with at least two key slabs (even slabs -> O_0, odd slabs -> O_1)
+      const bool use_o1 = (nq > 1) || (split && n_kv > 1);
 #pragma unroll
       for (int i = 0; i < 2; ++i) {
-        if (i >= nq) break;
-        const uint32_t itq = i == 0 ? it_q0 : it_q1;
-        ok = mbar_wait_warp(bar(kBarQFull + i), itq & 1u, abort_flag, 0x200 + i);
-        if (!ok) break;
-        // the epilogue of the previous item must have drained O_i before it is overwritten
-        ok = mbar_wait_warp(bar(kBarOEmpty + i), (itq & 1u) ^ 1u, abort_flag, 0x202 + i);
-        if (!ok) break;
+        if (i < nq) {
+          const uint32_t itq = i == 0 ? it_q0 : it_q1;
+          ok = mbar_wait_warp(bar(kBarQFull + i), itq & 1u, abort_flag, 0x200 + i);
+          if (!ok) break;
+        }
+        if (i == 0 || use_o1) {
+          // the epilogue of the previous item must have drained O_i before it is overwritten
+          const uint32_t ito = i == 0 ? it_o0 : it_o1;
+          ok = mbar_wait_warp(bar(kBarOEmpty + i), (ito & 1u) ^ 1u, abort_flag, 0x202 + i);
+          if (!ok) break;
+        }
       }
       if (!ok) break;
-      if (n_kv > 0) {
+      if (n_kv > 0 && split) {
+        // ---- split-KV item: one query slab (Q buffer 0); key slab j feeds tile (j & 1).
+        // Ring order (see the load warp): K_0, K_1, (V_0, K_2), (V_1, K_3), ..., V_{n-2}, V_{n-1}.
+        for (int j = 0; ok && j < 2 && j < n_kv; ++j) {
+          ok = mbar_wait_warp(bar(kBarPairFull + pair_g % kNumPairBars), (pair_g / kNumPairBars) & 1u, abort_flag, 0x230);
+          if (!ok) break;
+          ++pair_g;
+          const uint32_t slot = tile_g % kNumSlots;
+          ++tile_g;
+          tc_fence_after();
+          if (elect_one()) {
+            issue_qk(0, slot, nk_of(j), j);
+            tc_commit(bar(kBarSFull + j));
+            tc_commit(bar(kBarSlotEmpty + slot));
+          }
+          __syncwarp();
+        }
+        for (int j = 0; ok && j < n_kv; ++j) {
+          const int i = j & 1;
+          ok = mbar_wait_warp(bar(kBarPairFull + pair_g % kNumPairBars), (pair_g / kNumPairBars) & 1u, abort_flag, 0x231);
+          if (!ok) break;
+          ++pair_g;
+          const bool more = (j + 2 < n_kv);
+          const uint32_t vslot = tile_g % kNumSlots;
+          const uint32_t kslot = (tile_g + 1) % kNumSlots;
+          tile_g += more ? 2u : 1u;
+          const uint32_t cs = i == 0 ? cnt_s0 : cnt_s1;
+          const int nk_cur = nk_of(j);
+#if PSA_SPLIT_P
+          ok = mbar_wait_warp(bar(kBarPHalf + i), cs & 1u, abort_flag, 0x234 + i);
+          if (!ok) break;
+          tc_fence_after();
+          if (elect_one()) issue_pv_half(i, vslot, 0, j > 1, nk_cur);
+#endif
+          ok = mbar_wait_warp(bar(kBarPReady + i), cs & 1u, abort_flag, 0x232 + i);
+          if (!ok) break;
+          if (i == 0) ++cnt_s0; else ++cnt_s1;
+          tc_fence_after();
+          if (elect_one()) {
+#if PSA_SPLIT_P
+            issue_pv_half(i, vslot, 1, true, nk_cur);
+#else
+            issue_pv_half(i, vslot, 0, j > 1, nk_cur);
+            issue_pv_half(i, vslot, 1, true, nk_cur);
+#endif
+            tc_commit(bar(kBarSlotEmpty + vslot));
+            if (more) {
+              issue_qk(0, kslot, nk_of(j + 2), i);
+              tc_commit(bar(kBarSFull + i));
+              tc_commit(bar(kBarSlotEmpty + kslot));
+            } else {
+              tc_commit(bar(kBarOFull + i));
+            }
+          }
+          __syncwarp();
+        }
+        if (!ok) break;
+      } else if (n_kv > 0) {
         // first key slab: both S tiles
         {
           ok = mbar_wait_warp(bar(kBarPairFull + pair_g % kNumPairBars), (pair_g / kNumPairBars) & 1u, abort_flag, 0x210);
@@ -815,7 +897,7 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
 #pragma unroll
             for (int i = 0; i < 2; ++i) {
               if (i < nq) {
-                issue_qk(i, slot, g.n_sub == 1 ? g.n_last : kSlabTokens);
+                issue_qk(i, slot, nk_of(0), i);
                 tc_commit(bar(kBarSFull + i));
               }
             }
@@ -823,11 +905,9 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
           }
           __syncwarp();
         }
-        int sub = 0;  // slab index of key slab j inside its block
         for (int j = 0; ok && j < n_kv; ++j) {
-          const int nk_cur = (sub == g.n_sub - 1) ? g.n_last : kSlabTokens;
-          sub = (sub + 1 == g.n_sub) ? 0 : sub + 1;
-          const int nk_next = (sub == g.n_sub - 1) ? g.n_last : kSlabTokens;
+          const int nk_cur = nk_of(j);
+          const int nk_next = nk_of(j + 1);
           // V_j and (unless this is the last slab) K_{j+1} arrive under one barrier
           TRACE(2, j, 5);
           ok = mbar_wait_warp(bar(kBarPairFull + pair_g % kNumPairBars), (pair_g / kNumPairBars) & 1u, abort_flag, 0x211);
@@ -863,7 +943,7 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
 #endif
               if (i == nq - 1) tc_commit(bar(kBarSlotEmpty + vslot));
               if (more) {
-                issue_qk(i, kslot, nk_next);
+                issue_qk(i, kslot, nk_next, i);
                 tc_commit(bar(kBarSFull + i));
                 if (i == nq - 1) tc_commit(bar(kBarSlotEmpty + kslot));
               } else {
@@ -884,63 +964,94 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
       }
       ++it_q0;
       if (nq > 1) ++it_q1;
+      ++it_o0;
+      if (use_o1) ++it_o1;
     }
   }
   } else {
     asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
     // ======================================================================= softmax warps
-    const int qi = warp >> 2;                     // query slab handled by this warpgroup
+    const int qi = warp >> 2;                     // tile (S_i, O_i) handled by this warpgroup
     const int row = (warp & 3) * 32 + lane;       // row of the slab == TMEM lane
     const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
     const uint32_t tS = tmem + lane_addr + (uint32_t)qi * 128u;
     const uint32_t tO = tmem + lane_addr + 256u + (uint32_t)qi * 128u;
-    uint32_t it_q = 0, cnt_s = 0, kv_g = 0;
+    uint32_t it_o0 = 0, it_o1 = 0, cnt_s = 0, kv_g = 0;
     bool ok = true;
     const float neg_inf = __int_as_float(0xff800000);
+    float2* xchg = reinterpret_cast<float2*>(smem + kOffXchg);
 
     for (uint32_t n = 0; ok; ++n) {
       WorkItem wi;
       if (!next_item(n, wi)) break;
-      const int head = wi.x, qb = wi.y, sub0 = wi.w & 0xffff, nq = wi.w >> 16;
+      const int head = wi.x, qb = wi.y, sub0 = wi.w & 0xffff, nq = (wi.w >> 16) & 0xff;
+      const bool split = (wi.w >> 24) != 0;
       const int n_kv = wi.z * g.n_sub;
-      if (qi >= nq) {
-        kv_g += (uint32_t)n_kv;
-        continue;
-      }
+      const bool use_o1 = (nq > 1) || (split && n_kv > 1);
+      const bool active = (qi == 0) || use_o1;
       float m_ref = neg_inf;  // running reference maximum, scaled log2 domain
       float l = 0.f;          // running sum of exp2(s - m_ref)
-      int ksub = 0;           // slab index of key slab j inside its block
-      for (int j = 0; ok && j < n_kv; ++j, ++kv_g) {
-        const int nk = (ksub == g.n_sub - 1) ? g.n_last : kSlabTokens;
-        ksub = (ksub + 1 == g.n_sub) ? 0 : ksub + 1;
-        ok = mbar_wait_warp(bar(kBarSFull + qi), cnt_s & 1u, abort_flag, 0x300 + qi);
-        if (!ok) break;
-        ++cnt_s;
-        tc_fence_after();
-        TRACE(qi, j, 0);
-        // Read the slab's validity words first: shared memory is busy feeding the tensor core,
-        // so the load's latency is overlapped with the TMEM loads that follow.
-        const uint4 m = *reinterpret_cast<const uint4*>(meta + (kv_g % kMetaRing) * 8);
-        const uint32_t bh = bar(kBarPHalf + qi), br = bar(kBarPReady + qi);
+      if (active) {
+        // key slabs of this tile: all of them, or every second one in a split-KV item
+        const int j0 = split ? qi : 0, dj = split ? 2 : 1;
+        for (int j = j0; ok && j < n_kv; j += dj) {
+          const int nk = (j % g.n_sub == g.n_sub - 1) ? g.n_last : kSlabTokens;
+          ok = mbar_wait_warp(bar(kBarSFull + qi), cnt_s & 1u, abort_flag, 0x300 + qi);
+          if (!ok) break;
+          ++cnt_s;
+          tc_fence_after();
+          TRACE(qi, j, 0);
+          // Read the slab's validity words first: shared memory is busy feeding the tensor core,
+          // so the load's latency is overlapped with the TMEM loads that follow.
+          const uint4 m = *reinterpret_cast<const uint4*>(meta + ((kv_g + (uint32_t)j) % kMetaRing) * 8);
+          const uint32_t bh = bar(kBarPHalf + qi), br = bar(kBarPReady + qi);
 #ifdef PSA_TRACE
-        long long* tr = (blockIdx.x == 0 && n == 1 && j < 64 && (threadIdx.x & 127) == 0) ? g_trace + (qi * 64 + j) * 8 : nullptr;
+          long long* tr = (blockIdx.x == 0 && n == 1 && j < 64 && (threadIdx.x & 127) == 0) ? g_trace + (qi * 64 + j) * 8 : nullptr;
 #else
-        long long* tr = nullptr;
+          long long* tr = nullptr;
 #endif
-        if (nk == 128) softmax_slab<128>(tS, tO, m, j == 0, g.scale_log2, m_ref, l, bh, br, tr);
-        else if (nk == 112) softmax_slab<112>(tS, tO, m, j == 0, g.scale_log2, m_ref, l, bh, br, tr);
-        else if (nk == 96) softmax_slab<96>(tS, tO, m, j == 0, g.scale_log2, m_ref, l, bh, br, tr);
-        else softmax_slab<64>(tS, tO, m, j == 0, g.scale_log2, m_ref, l, bh, br, tr);
-        TRACE(qi, j, 4);
+          const bool first = (j == j0);
+          if (nk == 128) softmax_slab<128>(tS, tO, m, first, g.scale_log2, m_ref, l, bh, br, tr);
+          else if (nk == 112) softmax_slab<112>(tS, tO, m, first, g.scale_log2, m_ref, l, bh, br, tr);
+          else if (nk == 96) softmax_slab<96>(tS, tO, m, first, g.scale_log2, m_ref, l, bh, br, tr);
+          else softmax_slab<64>(tS, tO, m, first, g.scale_log2, m_ref, l, bh, br, tr);
+          TRACE(qi, j, 4);
+        }
       }
+      kv_g += (uint32_t)n_kv;
       if (!ok) break;
-      // ---- epilogue: out = O / l, lse = ln2 * (m_ref + log2 l)
-      ok = mbar_wait_warp(bar(kBarOFull + qi), it_q & 1u, abort_flag, 0x310 + qi);
+      const uint32_t par_o0 = it_o0 & 1u, par_o1 = it_o1 & 1u;
+      ++it_o0;
+      if (use_o1) ++it_o1;
+      if (!active) continue;
+
+      // ---- epilogue: out = O / l, lse = ln2 * (m_ref + log2 l).  In a split-KV item the two
+      // partial results (even / odd key slabs) of each row are merged by warpgroup 0, which can
+      // read both accumulators because they sit in the same TMEM lanes.
+      float scale0 = 1.f, scale1 = 0.f;   // weights of O_0 and O_1 in the merged output
+      if (split && qi == 1) {
+        xchg[row] = make_float2(m_ref, l);
+        named_bar_sync(3, 256);
+        continue;
+      }
+      ok = mbar_wait_warp(bar(kBarOFull + qi), (qi == 0 ? par_o0 : par_o1), abort_flag, 0x310 + qi);
       if (!ok) break;
-      ++it_q;
+      if (split && use_o1) {
+        ok = mbar_wait_warp(bar(kBarOFull + 1), par_o1, abort_flag, 0x312);
+        if (!ok) break;
+        named_bar_sync(3, 256);
+        const float2 other = xchg[row];
+        const float m_all = fmaxf(m_ref, other.x);
+        scale0 = (m_ref == neg_inf) ? 0.f : fast_exp2(m_ref - m_all);
+        scale1 = (other.x == neg_inf) ? 0.f : fast_exp2(other.x - m_all);
+        l = scale0 * l + scale1 * other.y;
+        m_ref = m_all;
+      }
       tc_fence_after();
       const bool empty = (n_kv == 0) || !(l > 0.f);
       const float inv = empty ? 0.f : 1.f / l;
+      scale0 *= inv;
+      scale1 *= inv;
       uint8_t* stage = smem + kOffQ + (uint32_t)qi * kSlabBytes;
 #pragma unroll
       for (int c4 = 0; c4 < 4; ++c4) {
@@ -952,13 +1063,24 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
 #pragma unroll
           for (int c = 0; c < 32; ++c) o[c] = 0u;
         }
+        if (split && use_o1) {   // qi == 0 here: add the odd-slab accumulator
+          uint32_t o1[32];
+          tc_ld32(tO + 128u + c4 * 32, o1);
+          tc_wait_ld();
+#pragma unroll
+          for (int c = 0; c < 32; ++c)
+            o[c] = __float_as_uint(__uint_as_float(o[c]) * scale0 + __uint_as_float(o1[c]) * scale1);
+        } else {
+#pragma unroll
+          for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * scale0);
+        }
 #pragma unroll
         for (int c8 = 0; c8 < 4; ++c8) {
           uint32_t w[4];
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
-            const float a = empty ? 0.f : __uint_as_float(o[c8 * 8 + 2 * e]) * inv;
-            const float b = empty ? 0.f : __uint_as_float(o[c8 * 8 + 2 * e + 1]) * inv;
+            const float a = empty ? 0.f : __uint_as_float(o[c8 * 8 + 2 * e]);
+            const float b = empty ? 0.f : __uint_as_float(o[c8 * 8 + 2 * e + 1]);
             w[e] = pack_bf16(a, b);
           }
           // 128-byte swizzle of the staging slab: 16-byte chunk index xor (row mod 8)
@@ -970,6 +1092,7 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
       }
       tc_fence_before();
       mbar_arrive(bar(kBarOEmpty + qi));
+      if (split && use_o1) mbar_arrive(bar(kBarOEmpty + 1));
       int t0, h0, w0, et, eh, ew, ntok, last;
       slab_origin(g, qb, sub0 + qi, t0, h0, w0);
       slab_shape(g, sub0 + qi, et, eh, ew, ntok, last);

@@ -155,6 +155,8 @@ def _sampled_rows(grid, tile, seed):
     ("wan14b_720p_b1x16x16", [2, 17, 31]),
     ("wan14b_720p_b3x8x16", [0, 13, 26]),
     ("hunyuan_720p", [1, 8, 15, 22]),
+    ("hunyuan_768p", [0, 11]),
+    ("hunyuan_768p_b6x8x8", [5, 23]),
     ("sweep_00", [0]), ("sweep_25", [3]), ("sweep_50", [5]), ("sweep_75", [7]), ("sweep_90", [39]),
     ("ragged_75", [0, 39]), ("ragged_dense", [20]),
 ])
