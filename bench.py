@@ -344,6 +344,80 @@ def run_ours(args, w):
         dist.destroy_process_group()
 
 
+def run_report(args):
+    """Times every committed workload (kernel-level: planning + attention kernels through psa_attn_fwd),
+    its all-covering (dense) counterpart and psa_mask_build, and writes a markdown table.  Inputs are
+    seeded N(0,1) bf16 tensors drawn on the device (timing does not depend on the values)."""
+    import ctypes
+    import torch
+    from paper_2609_37001_b200 import build
+    build.build()
+    from paper_2609_37001_b200 import binding as B
+    from paper_2609_37001_b200 import workloads as WL
+    peaks = load_peaks()
+    torch.cuda.set_device(0)
+    rows, dense_cache = [], {}
+    names = [n for n in WL.load_workloads() if not n.startswith("tiny")]
+    for name in names:
+        w = WL.workload(name)
+        T, H, W = w["grid"]
+        L, nh, tile = T * H * W, w["n_heads"], w["tile"]
+        params = [tuple(p) for p in w["head_params"]]
+        g = torch.Generator(device="cuda").manual_seed(w["seed"])
+        q, k, v = (torch.randn((nh, L, HEAD_DIM), device="cuda", generator=g).bfloat16() for _ in range(3))
+        out, lse = torch.empty_like(q), torch.empty((nh, L), dtype=torch.float32, device="cuda")
+
+        def timed(ps, iters):
+            for _ in range(2):
+                B.psa_attn_fwd(q, k, v, ps, w["grid"], tile, SCALE, out=out, lse=lse)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(iters):
+                B.psa_attn_fwd(q, k, v, ps, w["grid"], tile, SCALE, out=out, lse=lse)
+            e1.record()
+            torch.cuda.synchronize()
+            st, detail = B.psa_last_device_status()
+            if st != 0:
+                raise SystemExit(f"{name}: device status {st} {hex(detail)}")
+            return e0.elapsed_time(e1) / iters
+
+        flops, dflops = workload_flops(w)
+        ms = timed(params, 10 if flops < 6e13 else 4)
+        key = (tuple(w["grid"]), tuple(tile), nh)
+        if key not in dense_cache:
+            Tp, Hp, Wp = -(-T // tile[0]), -(-H // tile[1]), -(-W // tile[2])
+            dense_cache[key] = timed([(Tp, 0, 0, Hp * Wp, 0, 0)] * nh, 2)
+        dms = dense_cache[key]
+        nb, nnz = B.psa_mask_sizes(params, w["grid"], tile)
+        mo = (torch.empty((nh, nb, nb), dtype=torch.uint8, device="cuda"), torch.empty(nh * nb + 1, dtype=torch.int32, device="cuda"),
+              torch.empty(max(nnz, 1), dtype=torch.int32, device="cuda"))
+        prob = B.make_problem(nh, tile, 1.0, 0, 128)
+        margs = (B._params_array(params), ctypes.byref(prob), T, H, W, mo[0].data_ptr(), mo[1].data_ptr(), mo[2].data_ptr(), mo[2].numel(), None)
+        for _ in range(5):
+            B.lib().psa_mask_build(*margs)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(100):
+            B.lib().psa_mask_build(*margs)
+        e1.record()
+        torch.cuda.synchronize()
+        mb_us = 10.0 * e0.elapsed_time(e1)
+        mb_bytes = nh * (nb * nb + 4 * nb) + 4 + 4 * nnz
+        rows.append((name, "x".join(map(str, w["grid"])), L, nh, "x".join(map(str, tile)), w["tile_sparsity"], ms,
+                     flops / ms / 1e9, flops / ms / 1e9 / peaks["bf16_tflops"], dflops / ms / 1e9, dms, dms / ms,
+                     mb_us, mb_bytes / mb_us / 1e3))
+        del q, k, v, out, lse
+        torch.cuda.empty_cache()
+    lines = ["| workload | grid | tokens | heads | block | tile sparsity | ms/call | computed TFLOP/s | frac of measured peak | dense-equiv TFLOP/s | dense ms | speed-up vs dense | mask build us | mask build GB/s |",
+             "|---|---|---|---|---|---|---|---|---|---|---|---|---|---|"]
+    for r in rows:
+        lines.append("| %s | %s | %d | %d | %s | %.4f | %.3f | %.1f | %.3f | %.1f | %.2f | %.2f | %.1f | %.0f |" % r)
+    text = "\n".join(lines) + "\n"
+    with open(args.report, "w") as f:
+        f.write(text)
+    sys.stderr.write(text)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -352,7 +426,12 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="wan14b_720p")
     ap.add_argument("--quick", action="store_true", help="timed region only (no dense/e2e/CPU legs); for profiling")
+    ap.add_argument("--report", default=None, metavar="FILE.md",
+                    help="time every workload (PSA, dense, mask build) on one GPU and write a markdown table; no JSON line")
     args = ap.parse_args()
+    if args.report:
+        run_report(args)
+        return
     from paper_2609_37001_b200 import workloads as WL
     w = WL.workload(args.workload)
     if args.impl == "reference":

@@ -138,8 +138,9 @@ cudaError_t launch_mask_build(const HeadParamsArray& hp, const int* head_bases, 
     cudaError_t e = cudaFuncSetAttribute(mask_build_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
   }
-  // enough blocks per head to fill the machine about twice, at least 8 rows (one per warp) each
-  int blocks_per_head = (2 * n_sms + n_heads_here - 1) / n_heads_here;
+  // enough blocks per head to fill every SM's thread slots (8 blocks of 256 threads each),
+  // at least 8 rows (one per warp) per block
+  int blocks_per_head = (8 * n_sms + n_heads_here - 1) / n_heads_here;
   if (blocks_per_head < 1) blocks_per_head = 1;
   int rows_per_block = (g.NB + blocks_per_head - 1) / blocks_per_head;
   if (rows_per_block < 8) rows_per_block = 8;
