@@ -1,21 +1,27 @@
 // psa_attn_fwd for sm_100a: stripe-masked flash attention forward.
 //
-// One persistent CTA per SM walks a list of work items ordered by the number of
-// attended key blocks.  A work item is up to two 128-row query slabs of one query
-// block (PSABlock); both slabs share the block's key list (GetKVBlocks, Algorithm 2),
-// which the load warp enumerates in ascending block id straight from the six stripe
-// parameters (Algorithm 1) -- no mask or index list is read from memory.
+// One persistent CTA per SM draws work items from a global ticket; items are stored heaviest
+// first (by the number of attended key blocks), head-major.  A work item is up to two query
+// slabs (<= 128 rows each) of one query block (PSABlock); both slabs share the block's key
+// list (GetKVBlocks, Algorithm 2), which the load warp enumerates in ascending block id straight
+// from the six stripe parameters (Algorithm 1) -- no mask or index list is read from memory.
+// A single-slab item runs in split-KV mode: both softmax warpgroups work on that one slab, on
+// the even and the odd key slabs, and their partial results are merged in the epilogue.
 //
 // Roles (384 threads = 3 warpgroups):
-//   warps 0-3  softmax / correction / epilogue of query slab 0  (TMEM lanes 0..127)
-//   warps 4-7  the same for query slab 1
-//   warp  8    TMA loads: Q slabs once per item, K and V slabs through a 5-slot ring
+//   warps 0-3  softmax / correction / epilogue of tile 0 = (S0, O0)   (TMEM lanes 0..127)
+//   warps 4-7  the same for tile 1 = (S1, O1)
+//   warp  8    scheduler + TMA loads: Q slabs once per item, K and V slabs through a 5-slot ring
+//              (V_j travels with K_{j+1} under one barrier)
 //   warp  9    tcgen05.mma issue: S_i = Q_i K^T (SS form), O_i += P_i V (P read from TMEM)
 //   warps 10-11 idle; they only exist so that the third warpgroup can hand its registers
 //              to the softmax warpgroups (setmaxnreg)
 // TMEM (512 columns): S0 | S1 | O0 | O1, 128 fp32 columns each; the bf16 probabilities
-// P_i overwrite the first 64 columns of S_i.
+// P_i overwrite the first columns of S_i.  A key slab has 128 keys, or 112/96/64 for the last
+// slab of a block whose token count is not a multiple of 128.
 // Every wait is bounded; on expiry the CTA records a status word and unwinds.
+// Build-time knobs: PSA_SPLIT_P (publish P in two halves, default 1), PSA_EMU_PAIRS (share of
+// exponentials computed by a polynomial on the FMA pipe, default 0), PSA_TRACE (cycle stamps).
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -237,9 +243,6 @@ __device__ __forceinline__ void exp2_poly_pair(uint64_t x2, float& p0, float& p1
 #ifndef PSA_EMU_PAIRS
 #define PSA_EMU_PAIRS 0   // of every 4 pairs of probabilities, this many use exp2_poly_pair (0: all ex2.approx)
 #endif
-#ifndef PSA_MAX8
-#define PSA_MAX8 1        // eight row-max chains instead of four
-#endif
 #ifndef PSA_SPLIT_P
 #define PSA_SPLIT_P 1     // publish P in two halves of 64 keys
 #endif
@@ -253,16 +256,6 @@ __device__ __forceinline__ void named_bar_sync(int id, int nthreads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
 }
 
-// Shared-memory matrix descriptor, 128-byte swizzle, sm_100 version field.
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
-  uint64_t d = 0;
-  d |= (uint64_t)((addr >> 4) & 0x3FFFu);
-  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
-  d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
-  d |= 1ull << 46;  // descriptor version
-  d |= 2ull << 61;  // 128-byte swizzle
-  return d;
-}
 // Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N columns (multiple of 16); A is K-major.
 __host__ __device__ constexpr uint32_t instr_desc(bool b_mn_major, uint32_t n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((n >> 3) << 17) | ((128u >> 4) << 24);
@@ -411,7 +404,6 @@ __device__ __forceinline__ void softmax_slab(uint32_t tS, uint32_t tO, const uin
       if (!((v[c >> 5] >> (c & 31)) & 1u)) s[c] = 0xff800000u;
   }
   STAMP(7);
-#if PSA_MAX8
   // eight independent chains (NK is a multiple of 16): shorter dependency depth
   float a[8];
 #pragma unroll
@@ -422,18 +414,6 @@ __device__ __forceinline__ void softmax_slab(uint32_t tS, uint32_t tO, const uin
     for (int i = 0; i < 8; ++i) a[i] = max3(a[i], __uint_as_float(s[c + 2 * i]), __uint_as_float(s[c + 2 * i + 1]));
   }
   const float ms = fmaxf(fmaxf(max3(a[0], a[1], a[2]), max3(a[3], a[4], a[5])), fmaxf(a[6], a[7])) * scale_log2;
-#else
-  float a0 = neg_inf, a1 = neg_inf, a2 = neg_inf, a3 = neg_inf;
-#pragma unroll
-  for (int c = 0; c < NK; c += 8) {
-    a0 = max3(a0, __uint_as_float(s[c]), __uint_as_float(s[c + 1]));
-    a1 = max3(a1, __uint_as_float(s[c + 2]), __uint_as_float(s[c + 3]));
-    a2 = max3(a2, __uint_as_float(s[c + 4]), __uint_as_float(s[c + 5]));
-    a3 = max3(a3, __uint_as_float(s[c + 6]), __uint_as_float(s[c + 7]));
-  }
-  const float ms = fmaxf(fmaxf(a0, a1), fmaxf(a2, a3)) * scale_log2;
-#endif
-  STAMP(5);   // (overwritten later by the half-way stamp when tracing the split; read before)
   if (first) {
     m_ref = ms;  // first slab of the item: nothing accumulated yet
   } else {
