@@ -123,9 +123,13 @@ int psa_attn_fwd_noalloc(const void* q, const void* k, const void* v, void* out,
                          const psa_head_params* head_params, const psa_problem* prob,
                          int T, int H, int W, void* stream, int32_t* status_detail);
 
-/* The same call for HOST tensors: copies q, k, v (host, pinned for speed) into the
- * caller's device staging buffers d_q, d_k, d_v, runs psa_attn_fwd into d_out / d_lse
- * and copies the results to out / lse (host), all on `stream`, then synchronises it.
+/* The same call for HOST tensors: copies q, k, v (host; pinned memory is needed for the
+ * copies to overlap) into the caller's device staging buffers d_q, d_k, d_v, runs
+ * psa_attn_fwd into d_out / d_lse and copies the results to out / lse (host), ordered
+ * after the work already on `stream`, then synchronises `stream`.  When heads are the
+ * outermost dimension of the layout the call is pipelined over up to 8 chunks of heads on
+ * two internal helper streams: the next chunk is copied in and the previous one copied out
+ * while a chunk computes.
  * Each staging buffer must hold the full strided extent of its tensor:
  * (n_heads-1)*stride_head + (L-1)*stride_token + head_dim elements. */
 int psa_attn_fwd_host(const void* q, const void* k, const void* v, void* out, float* lse,

@@ -192,6 +192,30 @@ int encode_maps(TensorMaps* tm, const void* q, const void* k, const void* v, voi
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// ---- helper streams of psa_attn_fwd_host (one set per device, created on first use) ----------
+constexpr int kHostChunks = 8;
+struct HostPipe {
+  bool ready = false;
+  cudaStream_t h2d = nullptr, d2h = nullptr;
+  cudaEvent_t ev_start = nullptr, ev_end = nullptr, ev_in[kHostChunks] = {}, ev_done[kHostChunks] = {};
+};
+HostPipe g_pipe[kMaxDevices];
+
+HostPipe* host_pipe(int dev) {   // caller holds g_mu; returns nullptr if the streams cannot be created
+  HostPipe& p = g_pipe[dev];
+  if (p.ready) return &p;
+  if (cudaStreamCreateWithFlags(&p.h2d, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+  if (cudaStreamCreateWithFlags(&p.d2h, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+  if (cudaEventCreateWithFlags(&p.ev_start, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+  if (cudaEventCreateWithFlags(&p.ev_end, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+  for (int i = 0; i < kHostChunks; ++i) {
+    if (cudaEventCreateWithFlags(&p.ev_in[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    if (cudaEventCreateWithFlags(&p.ev_done[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
+  }
+  p.ready = true;
+  return &p;
+}
+
 // ---- scratch of psa_attn_fwd_noalloc ------------------------------------------------------
 // Layout: 16 int32 header words (status, detail, scheduler ticket), kMaxHeads head parameter
 // records, then up to kNoAllocMaxItems work items.  It lives in every GPU that loads the
@@ -420,20 +444,71 @@ int psa_attn_fwd_noalloc(const void* q, const void* k, const void* v, void* out,
 int psa_attn_fwd_host(const void* q, const void* k, const void* v, void* out, float* lse, void* d_q, void* d_k, void* d_v,
                       void* d_out, float* d_lse, const psa_head_params* head_params, const psa_problem* prob, int T, int H,
                       int W, void* stream) {
-  if (!prob || !q || !k || !v || !out || !lse || !d_q || !d_k || !d_v || !d_out || !d_lse) return PSA_ERR_INVALID_ARG;
+  if (!prob || !q || !k || !v || !out || !lse || !d_q || !d_k || !d_v || !d_out || !d_lse || !head_params)
+    return PSA_ERR_INVALID_ARG;
   if (T < 1 || H < 1 || W < 1 || prob->n_heads < 1) return PSA_ERR_INVALID_ARG;
   const long long L = (long long)T * H * W;
-  const size_t elems = (size_t)(prob->n_heads - 1) * prob->stride_head + (size_t)(L - 1) * prob->stride_token + prob->head_dim;
-  const size_t bytes = elems * 2;
+  const size_t head_span = (size_t)(L - 1) * prob->stride_token + prob->head_dim;  // elements one head touches
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (cudaMemcpyAsync(d_q, q, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return PSA_ERR_CUDA;
-  if (cudaMemcpyAsync(d_k, k, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return PSA_ERR_CUDA;
-  if (cudaMemcpyAsync(d_v, v, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return PSA_ERR_CUDA;
-  const int rc = psa_attn_fwd(d_q, d_k, d_v, d_out, d_lse, head_params, prob, T, H, W, stream);
-  if (rc != PSA_OK) return rc;
-  if (cudaMemcpyAsync(out, d_out, bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return PSA_ERR_CUDA;
-  if (cudaMemcpyAsync(lse, d_lse, sizeof(float) * (size_t)prob->n_heads * L, cudaMemcpyDeviceToHost, st) != cudaSuccess)
-    return PSA_ERR_CUDA;
+
+  // Heads are independent problems: when they are the outermost dimension of the layout the
+  // call is pipelined over chunks of heads -- chunk c+1 is copied in and chunk c-1 copied out
+  // while chunk c computes (two helper streams per device, created on first use).
+  const bool head_major = prob->n_heads == 1 || (size_t)prob->stride_head >= head_span;
+  int dev = 0;
+  HostPipe* pipe = nullptr;
+  if (head_major && prob->n_heads >= 2 && cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < kMaxDevices) {
+    std::lock_guard<std::mutex> lock(g_mu);
+    pipe = host_pipe(dev);
+  }
+  if (!pipe) {
+    const size_t bytes = ((size_t)(prob->n_heads - 1) * prob->stride_head + head_span) * 2;
+    if (cudaMemcpyAsync(d_q, q, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return PSA_ERR_CUDA;
+    if (cudaMemcpyAsync(d_k, k, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return PSA_ERR_CUDA;
+    if (cudaMemcpyAsync(d_v, v, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return PSA_ERR_CUDA;
+    const int rc = psa_attn_fwd(d_q, d_k, d_v, d_out, d_lse, head_params, prob, T, H, W, stream);
+    if (rc != PSA_OK) return rc;
+    if (cudaMemcpyAsync(out, d_out, bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return PSA_ERR_CUDA;
+    if (cudaMemcpyAsync(lse, d_lse, sizeof(float) * (size_t)prob->n_heads * L, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+      return PSA_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return PSA_ERR_CUDA;
+    return PSA_OK;
+  }
+
+  const int n_chunks = prob->n_heads < kHostChunks ? prob->n_heads : kHostChunks;
+  const int per = (prob->n_heads + n_chunks - 1) / n_chunks;
+  // everything enqueued on `stream` before this call precedes the first copy
+  if (cudaEventRecord(pipe->ev_start, st) != cudaSuccess) return PSA_ERR_CUDA;
+  if (cudaStreamWaitEvent(pipe->h2d, pipe->ev_start, 0) != cudaSuccess) return PSA_ERR_CUDA;
+  if (cudaStreamWaitEvent(pipe->d2h, pipe->ev_start, 0) != cudaSuccess) return PSA_ERR_CUDA;
+  int c = 0;
+  for (int h0 = 0; h0 < prob->n_heads; h0 += per, ++c) {
+    const int nh = prob->n_heads - h0 < per ? prob->n_heads - h0 : per;
+    const size_t off = (size_t)h0 * prob->stride_head;                       // elements
+    const size_t bytes = ((size_t)(nh - 1) * prob->stride_head + head_span) * 2;
+    const uint16_t *hq = static_cast<const uint16_t*>(q) + off, *hk = static_cast<const uint16_t*>(k) + off,
+                   *hv = static_cast<const uint16_t*>(v) + off;
+    uint16_t *dq = static_cast<uint16_t*>(d_q) + off, *dk = static_cast<uint16_t*>(d_k) + off,
+             *dv = static_cast<uint16_t*>(d_v) + off, *dout = static_cast<uint16_t*>(d_out) + off;
+    if (cudaMemcpyAsync(dq, hq, bytes, cudaMemcpyHostToDevice, pipe->h2d) != cudaSuccess) return PSA_ERR_CUDA;
+    if (cudaMemcpyAsync(dk, hk, bytes, cudaMemcpyHostToDevice, pipe->h2d) != cudaSuccess) return PSA_ERR_CUDA;
+    if (cudaMemcpyAsync(dv, hv, bytes, cudaMemcpyHostToDevice, pipe->h2d) != cudaSuccess) return PSA_ERR_CUDA;
+    if (cudaEventRecord(pipe->ev_in[c], pipe->h2d) != cudaSuccess) return PSA_ERR_CUDA;
+    if (cudaStreamWaitEvent(st, pipe->ev_in[c], 0) != cudaSuccess) return PSA_ERR_CUDA;
+    psa_problem sub = *prob;
+    sub.n_heads = nh;
+    const int rc = psa_attn_fwd(dq, dk, dv, dout, d_lse + (size_t)h0 * L, head_params + h0, &sub, T, H, W, stream);
+    if (rc != PSA_OK) return rc;
+    if (cudaEventRecord(pipe->ev_done[c], st) != cudaSuccess) return PSA_ERR_CUDA;
+    if (cudaStreamWaitEvent(pipe->d2h, pipe->ev_done[c], 0) != cudaSuccess) return PSA_ERR_CUDA;
+    if (cudaMemcpyAsync(static_cast<uint16_t*>(out) + off, dout, bytes, cudaMemcpyDeviceToHost, pipe->d2h) != cudaSuccess)
+      return PSA_ERR_CUDA;
+    if (cudaMemcpyAsync(lse + (size_t)h0 * L, d_lse + (size_t)h0 * L, sizeof(float) * (size_t)nh * L, cudaMemcpyDeviceToHost,
+                        pipe->d2h) != cudaSuccess)
+      return PSA_ERR_CUDA;
+  }
+  if (cudaEventRecord(pipe->ev_end, pipe->d2h) != cudaSuccess) return PSA_ERR_CUDA;
+  if (cudaStreamWaitEvent(st, pipe->ev_end, 0) != cudaSuccess) return PSA_ERR_CUDA;
   if (cudaStreamSynchronize(st) != cudaSuccess) return PSA_ERR_CUDA;
   return PSA_OK;
 }

@@ -164,3 +164,27 @@ def test_full_size_workloads_sampled_rows(B, name, heads):
     w = WL.workload(name)
     _run_and_check(B, w["head_params"], w["grid"], w["tile"], w["seed"],
                    rows_per_head=_sampled_rows(w["grid"], w["tile"], w["seed"]), heads_to_check=heads)
+
+
+@pytest.mark.parametrize("pinned", [True, False])
+def test_host_tensor_entry_point_matches_device_call(B, pinned):
+    """psa_attn_fwd_host (copies in, pipelined over head chunks, copies out) gives the device call's bits,
+    with more heads than chunks and with fewer heads than chunks, from pinned and from pageable memory."""
+    for nh, grid, tile in ((11, (4, 16, 16), (1, 16, 16)), (3, (3, 15, 32), (1, 15, 16))):
+        T, H, W = grid
+        L = T * H * W
+        params = [(1 + (h % 3), (h % 3) - 1, [INF, 2, 3][h % 3], 1 + (h % 2), 0, [INF, 3][h % 2]) for h in range(nh)]
+        bits = {n: WL.tensor_bits(0x7A + nh, n, nh, L, threads=1) for n in ("q", "k", "v")}
+        host = {n: torch.from_numpy(bits[n].view(np.int16)).view(torch.bfloat16) for n in bits}
+        dev = {n: host[n].cuda() for n in host}
+        ref_out, ref_lse = B.psa_attn_fwd(dev["q"], dev["k"], dev["v"], params, grid, tile, SCALE)
+        assert B.psa_last_device_status()[0] == 0
+        hq, hk, hv = (host[n].pin_memory() if pinned else host[n].clone() for n in ("q", "k", "v"))
+        hout = torch.full_like(hq, float("nan"))
+        hlse = torch.full((nh, L), float("nan"), dtype=torch.float32)
+        if pinned:
+            hout, hlse = hout.pin_memory(), hlse.pin_memory()
+        staging = tuple(torch.empty_like(dev["q"]) for _ in range(4)) + (torch.empty((nh, L), dtype=torch.float32, device="cuda"),)
+        B.psa_attn_fwd_host(hq, hk, hv, hout, hlse, staging, params, grid, tile, SCALE)
+        assert torch.equal(hout.view(torch.int16), ref_out.cpu().view(torch.int16))
+        assert torch.equal(hlse.view(torch.int32), ref_lse.cpu().view(torch.int32))
