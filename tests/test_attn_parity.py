@@ -188,3 +188,18 @@ def test_host_tensor_entry_point_matches_device_call(B, pinned):
         B.psa_attn_fwd_host(hq, hk, hv, hout, hlse, staging, params, grid, tile, SCALE)
         assert torch.equal(hout.view(torch.int16), ref_out.cpu().view(torch.int16))
         assert torch.equal(hlse.view(torch.int32), ref_lse.cpu().view(torch.int32))
+
+
+def test_more_heads_than_one_launch_carries(B):
+    """130 heads: the library splits the call into launches of at most 128 heads."""
+    grid, tile, nh = (2, 16, 16), (1, 16, 16), 130
+    L = 2 * 16 * 16
+    params = [((h % 2) + 1, (h % 3) - 1, INF, 1, 0, INF) for h in range(nh)]
+    bits = {n: WL.tensor_bits(0x7B, n, nh, L) for n in ("q", "k", "v")}
+    q, k, v = (_to_dev(bits[n]) for n in ("q", "k", "v"))
+    out, lse = B.psa_attn_fwd(q, k, v, params, grid, tile, SCALE)
+    assert B.psa_last_device_status()[0] == 0
+    for hd in (0, 1, 63, 127, 128, 129):
+        qf, kf, vf = (O.bf16_bits_to_f64(bits[n][hd]) for n in ("q", "k", "v"))
+        ro, rl = O.attention(qf, kf, vf, params[hd], *grid, tile, SCALE)
+        _compare(_bf16_to_f64(out[hd]), lse[hd].cpu().numpy().astype(np.float64), ro, rl, f"head {hd}")
