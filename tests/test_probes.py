@@ -122,3 +122,31 @@ def test_device_errors_are_codes_not_faults(B):
     assert e.value.status == B.PSA_ERR_INVALID_ARG
     with pytest.raises(ValueError):
         B.psa_attn_fwd(q.cpu(), q.cpu(), q.cpu(), [(1, 0, 0, 1, 0, 0)], (1, 16, 16), (1, 16, 16), SCALE)
+
+
+@pytest.mark.parametrize("tile", [(1, 16, 16), (1, 8, 16), (3, 8, 16), (1, 15, 16)])
+def test_scores_growing_along_the_keys_force_rescales(B, tile):
+    """Keys are scaled so that every later key slab raises each row's maximum by far more than the lazy
+    rescale threshold: the running reference maximum moves, and the output accumulator is rescaled, at
+    (almost) every slab.  A decreasing variant checks the opposite extreme (never after the first slab)."""
+    grid = (6, 16 if tile[1] != 15 else 15, 16)
+    T, H, W = grid
+    L, nh = T * H * W, 2
+    rng = np.random.default_rng(0x94)
+    base = rng.standard_normal((L, 128)).astype(np.float32)
+    ramp = np.linspace(0.2, 6.0, L, dtype=np.float32)[:, None]
+    q = WL.f32_to_bf16_bits(rng.standard_normal((nh, L, 128)).astype(np.float32))
+    v = WL.f32_to_bf16_bits(rng.standard_normal((nh, L, 128)).astype(np.float32))
+    k = WL.f32_to_bf16_bits(np.stack([base * ramp, base * ramp[::-1]]))
+    dev = [torch.from_numpy(x.view(np.int16)).cuda().view(torch.bfloat16) for x in (q, k, v)]
+    Tp, Hp, Wp = O.block_grid(T, H, W, tile)
+    params = [(Tp, 0, INF, Hp * Wp, 0, INF), (Tp, 0, INF, Hp * Wp, 0, INF)]
+    out, lse = B.psa_attn_fwd(*dev, params, grid, tile, SCALE)
+    assert B.psa_last_device_status()[0] == 0
+    out_h = O.bf16_bits_to_f64(out.view(torch.int16).cpu().numpy().view(np.uint16))
+    lse_h = lse.cpu().numpy().astype(np.float64)
+    for hd in range(nh):
+        ro, rl = O.dense_attention(*(O.bf16_bits_to_f64(x[hd]) for x in (q, k, v)), SCALE)
+        err = np.abs(out_h[hd] - ro)
+        assert err.max() <= 2e-2 and err.mean() <= 2e-3, (hd, err.max(), err.mean())
+        assert np.abs(lse_h[hd] - rl).max() <= 1e-3, (hd, np.abs(lse_h[hd] - rl).max(), np.abs(rl).max())
