@@ -310,3 +310,33 @@ def dense_flops(L: int, d: int, heads: int) -> float:
 
 def computed_flops(head_params: Sequence[Params], T: int, H: int, W: int, tile: Tile, d: int) -> float:
     return 4.0 * d * sum(attended_pairs(p, T, H, W, tile) for p in head_params)
+
+
+# --------------------------------------------------------------------------- #
+# PSA-Search for one head (Algorithm 3)
+# --------------------------------------------------------------------------- #
+def search_losses(q: np.ndarray, k: np.ndarray, v: np.ndarray, candidates: Sequence[Params],
+                  T: int, H: int, W: int, tile: Tile, scale: float) -> np.ndarray:
+    """Inner loop of Algorithm 3 for one head: Loss(M) = L2Loss(PSA(h, M), FullAttn(h)) for every
+    candidate mask M.  The paper does not spell the loss out; it is taken as the mean squared
+    difference over all output elements.  q, k, v: float64 [L, d].  Returns float64[len(candidates)]."""
+    full, _ = dense_attention(q, k, v, scale)
+    losses = np.zeros(len(candidates), dtype=np.float64)
+    for c, p in enumerate(candidates):
+        out, _ = attention(q, k, v, p, T, H, W, tile, scale)
+        losses[c] = np.mean((out - full) ** 2)
+    return losses
+
+
+def search_select(losses: Sequence[float], sparsities: Sequence[float], alpha: float) -> int:
+    """Selection of Algorithm 3 for one head, step by step: sort the candidates by loss (ascending,
+    ties by candidate index); start from the lowest-loss candidate; scan the sorted list and, among
+    those whose loss does not exceed alpha, replace the current best whenever a candidate is strictly
+    sparser.  Returns the index of the chosen candidate."""
+    order = sorted(range(len(losses)), key=lambda i: (losses[i], i))
+    best = order[0]
+    for i in order:
+        if losses[i] <= alpha:
+            if sparsities[i] > sparsities[best]:
+                best = i
+    return best
