@@ -61,7 +61,7 @@ def test_losses_against_direct_formulas():
              (1, 0, INF, Hp * Wp, 0, INF),       # same frame block only
              (1, 0, INF, 1, 0, INF)]             # same block only
     losses = O.search_losses(q, k, v, cands, T, H, W, tile, scale)
-    assert losses[0] == 0.0
+    assert losses[0] < 1e-28          # same numbers up to summation order
     # written out with a boolean mask and a library softmax, then the mean of squares
     import torch
     tq, tk, tv = (torch.from_numpy(x)[None, None] for x in (q, k, v))
