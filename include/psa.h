@@ -137,6 +137,31 @@ int psa_attn_fwd_host(const void* q, const void* k, const void* v, void* out, fl
                       const psa_head_params* head_params, const psa_problem* prob,
                       int T, int H, int W, void* stream);
 
+/* PSA-Search for ONE head (Appendix C, Algorithm 3).
+ *
+ * psa_search_losses: the inner loop -- Loss(M) = L2Loss(PSA(h, M), FullAttn(h)) for every candidate
+ * mask M.  All n_cand candidates and full attention (an all-covering mask) run in one launch of the
+ * stripe attention kernel on the same q, k, v; then loss[c] = mean over all L*128 output elements of
+ * (out_c - out_full)^2 (the paper does not spell the loss out; mean squared difference is the reading
+ * taken).  q, k, v: device bf16, ONE head, element (token, c) at token*stride_token + c (prob->n_heads
+ * and stride_head are ignored; tile, scale, head_dim as for psa_attn_fwd).  candidates: host.
+ * scratch: device, 256-byte aligned, psa_search_scratch_bytes(n_cand, T, H, W) bytes (holds every
+ * candidate's output).  losses: device fp32 [n_cand].  Asynchronous on `stream`.
+ *
+ * psa_search_select: the selection -- sort by loss ascending (ties by index), start from the
+ * lowest-loss candidate, and among candidates with loss <= alpha move to any strictly sparser one.
+ * losses, sparsity: host arrays of n entries (sparsity = excluded fraction of block pairs, e.g. from
+ * psa_mask_sizes).  Returns the chosen index (>= 0) or a negative psa_status.  Pure host code.
+ *
+ * psa_search_select_at_sparsity: the second interface of Section 3.3 -- for a target sparsity, the
+ * candidate of minimal loss among those with sparsity >= target (ties by index); PSA_ERR_CAPACITY
+ * when no candidate is that sparse.  Pure host code. */
+int64_t psa_search_scratch_bytes(int n_cand, int T, int H, int W);
+int psa_search_losses(const void* q, const void* k, const void* v, const psa_head_params* candidates, int n_cand,
+                      const psa_problem* prob, int T, int H, int W, void* scratch, float* losses, void* stream);
+int psa_search_select(const float* losses, const float* sparsity, int n, float alpha);
+int psa_search_select_at_sparsity(const float* losses, const float* sparsity, int n, float target);
+
 /* Synchronises the current device, then returns the status word the last psa_attn_fwd
  * on it left behind: PSA_OK, or PSA_ERR_TIMEOUT if a bounded wait inside the kernel
  * expired (outputs are then undefined).  *detail (optional, host) receives a

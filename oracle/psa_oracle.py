@@ -340,3 +340,16 @@ def search_select(losses: Sequence[float], sparsities: Sequence[float], alpha: f
             if sparsities[i] > sparsities[best]:
                 best = i
     return best
+
+
+def search_select_at_sparsity(losses: Sequence[float], sparsities: Sequence[float], target: float) -> int:
+    """Second interface of PSA-Search (Section 3.3): given a target sparsity, the candidate with minimal
+    loss among those at least that sparse (ties by candidate index); -1 when no candidate reaches the
+    target."""
+    best = -1
+    for i in range(len(losses)):
+        if sparsities[i] >= target:
+            if best < 0 or losses[i] < losses[best]:
+                best = i
+    return best
+

@@ -64,6 +64,14 @@ def lib() -> ctypes.CDLL:
         L.psa_attn_fwd_host.argtypes = [vp] * 10 + [hp, pp, i32, i32, i32, vp]
         L.psa_attn_fwd_noalloc.argtypes = [vp, vp, vp, vp, vp, hp, pp, i32, i32, i32, vp, ctypes.POINTER(ctypes.c_int32)]
         L.psa_attn_fwd_noalloc.restype = ctypes.c_int
+        L.psa_search_scratch_bytes.argtypes = [i32, i32, i32, i32]
+        L.psa_search_scratch_bytes.restype = ctypes.c_int64
+        L.psa_search_losses.argtypes = [vp, vp, vp, hp, i32, pp, i32, i32, i32, vp, vp, vp]
+        L.psa_search_losses.restype = ctypes.c_int
+        L.psa_search_select.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_float), i32, ctypes.c_float]
+        L.psa_search_select.restype = ctypes.c_int
+        L.psa_search_select_at_sparsity.argtypes = L.psa_search_select.argtypes
+        L.psa_search_select_at_sparsity.restype = ctypes.c_int
         L.psa_last_device_status.argtypes = [ctypes.POINTER(ctypes.c_int32)]
         L.psa_shutdown.argtypes = []
         L.psa_selftest_wait_timeout.argtypes = [i32, vp]
@@ -225,6 +233,72 @@ def psa_attn_fwd_host(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, out: to
                                    d_q.data_ptr(), d_k.data_ptr(), d_v.data_ptr(), d_out.data_ptr(),
                                    d_lse.data_ptr(), _params_array(head_params), ctypes.byref(prob), T, H, W,
                                    _stream_ptr(stream)), "psa_attn_fwd_host")
+
+
+def psa_search_scratch_bytes(n_cand: int, grid: Sequence[int]) -> int:
+    """Bytes of device scratch psa_search_losses needs for ``n_cand`` candidates on this token grid."""
+    T, H, W = (int(x) for x in grid)
+    n = int(lib().psa_search_scratch_bytes(int(n_cand), T, H, W))
+    if n < 0:
+        _check(n, "psa_search_scratch_bytes")
+    return n
+
+
+def psa_search_losses(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, candidates, grid: Sequence[int],
+                      tile: Sequence[int], scale: float, scratch: Optional[torch.Tensor] = None,
+                      stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """Inner loop of PSA-Search for one head (Algorithm 3): q, k, v are bf16 [L, 128] device tensors of
+    that head, ``candidates`` a sequence of six-integer masks.  Returns the fp32 loss of every candidate
+    against full attention (device tensor).  ``scratch`` (uint8, psa_search_scratch_bytes long) is
+    allocated when not given."""
+    _require_cuda(q, k, v)
+    L, d = q.shape
+    T, H, W = (int(x) for x in grid)
+    if L != T * H * W or k.shape != q.shape or v.shape != q.shape:
+        raise ValueError("shape mismatch")
+    if q.stride() != k.stride() or q.stride() != v.stride() or q.stride(1) != 1:
+        raise ValueError("q, k, v must share strides with a contiguous last dimension")
+    n_cand = len(candidates)
+    need = psa_search_scratch_bytes(n_cand, grid)
+    if scratch is None:
+        scratch = torch.empty(need, dtype=torch.uint8, device=q.device)
+    if scratch.numel() * scratch.element_size() < need or not scratch.is_contiguous():
+        raise ValueError("scratch too small")
+    losses = torch.empty(n_cand, dtype=torch.float32, device=q.device)
+    prob = make_problem(1, tile, scale, 0, q.stride(0), d)
+    _check(lib().psa_search_losses(q.data_ptr(), k.data_ptr(), v.data_ptr(), _params_array(candidates), n_cand,
+                                   ctypes.byref(prob), T, H, W, scratch.data_ptr(), losses.data_ptr(),
+                                   _stream_ptr(stream)), "psa_search_losses")
+    return losses
+
+
+def psa_search_select(losses: Sequence[float], sparsity: Sequence[float], alpha: float) -> int:
+    """Selection step of PSA-Search (Algorithm 3) on host arrays; returns the chosen candidate's index."""
+    n = len(losses)
+    if len(sparsity) != n:
+        raise ValueError("losses and sparsity differ in length")
+    la = (ctypes.c_float * n)(*[float(x) for x in losses])
+    sa = (ctypes.c_float * n)(*[float(x) for x in sparsity])
+    r = int(lib().psa_search_select(la, sa, n, float(alpha)))
+    if r < 0:
+        _check(r, "psa_search_select")
+    return r
+
+
+def psa_search_select_at_sparsity(losses: Sequence[float], sparsity: Sequence[float], target: float) -> int:
+    """Second interface of PSA-Search: minimal-loss candidate among those at least ``target`` sparse;
+    -1 when none is."""
+    n = len(losses)
+    if len(sparsity) != n:
+        raise ValueError("losses and sparsity differ in length")
+    la = (ctypes.c_float * n)(*[float(x) for x in losses])
+    sa = (ctypes.c_float * n)(*[float(x) for x in sparsity])
+    r = int(lib().psa_search_select_at_sparsity(la, sa, n, float(target)))
+    if r == -3:  # PSA_ERR_CAPACITY: no candidate reaches the target
+        return -1
+    if r < 0:
+        _check(r, "psa_search_select_at_sparsity")
+    return r
 
 
 def psa_last_device_status() -> Tuple[int, int]:

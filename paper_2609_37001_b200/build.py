@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libpsa.so")
-SOURCES = ["psa_host.cu", "psa_mask_build.cu", "psa_attn_sm100.cu"]
+SOURCES = ["psa_host.cu", "psa_mask_build.cu", "psa_attn_sm100.cu", "psa_search.cu"]
 HEADERS = [os.path.join(CSRC, "psa_common.cuh"), os.path.join(ROOT, "include", "psa.h")]
 
 

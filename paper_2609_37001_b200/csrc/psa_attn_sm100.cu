@@ -336,6 +336,7 @@ struct AttnParams {
   int* ws_header;
   float* lse;     // already offset to the first head of this launch
   int n_items;
+  int shared_qkv; // 1: every head reads head 0 of q, k, v (candidate masks of one head, PSA-Search)
 };
 
 struct TensorMaps {
@@ -588,6 +589,7 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
       if (wi.x < 0) break;
       const int head = wi.x, qb = wi.y, sub0 = wi.w & 0xffff, nq = (wi.w >> 16) & 0xff;
       const int lag = (wi.w >> 24) ? 2 : 1;   // V_j travels with K_{j+lag} (2 in split-KV mode)
+      const int head_ld = prm.shared_qkv ? 0 : head;   // head coordinate of the q, k, v loads
       const psa_head_params p = prm.hp_dev[head];
       const int tq = qb / g.Sp, sq = qb % g.Sp;
       // attended key-block coordinates of this query block, one bit per block coordinate
@@ -615,8 +617,8 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
           slab_shape(g, sub0 + i, et, eh, ew, ntok, last);
           const uint32_t dst = sbase + kOffQ + (uint32_t)i * kSlabBytes;
           mbar_expect_tx(bar(kBarQFull + i), (uint32_t)ntok * 256u);
-          tma_load_5d(dst, &tms.q[last], bar(kBarQFull + i), 0, w0, h0, t0, head);
-          tma_load_5d(dst + kHalfBytes, &tms.q[last], bar(kBarQFull + i), 64, w0, h0, t0, head);
+          tma_load_5d(dst, &tms.q[last], bar(kBarQFull + i), 0, w0, h0, t0, head_ld);
+          tma_load_5d(dst + kHalfBytes, &tms.q[last], bar(kBarQFull + i), 64, w0, h0, t0, head_ld);
         }
         if (i == 0) ++it_q0; else ++it_q1;
       }
@@ -672,12 +674,12 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
                   mbar_expect_tx(pb, (uint32_t)((with_v ? antok : 0) + ntok) * 256u);
                   if (with_v) {
                     const uint32_t dv = sbase + kOffRing + v_slot * kSlabBytes;
-                    tma_load_5d(dv, &tms.v[alast], pb, 0, aw0, ah0, at0, head);
-                    tma_load_5d(dv + kHalfBytes, &tms.v[alast], pb, 64, aw0, ah0, at0, head);
+                    tma_load_5d(dv, &tms.v[alast], pb, 0, aw0, ah0, at0, head_ld);
+                    tma_load_5d(dv + kHalfBytes, &tms.v[alast], pb, 64, aw0, ah0, at0, head_ld);
                   }
                   const uint32_t dk = sbase + kOffRing + k_slot * kSlabBytes;
-                  tma_load_5d(dk, &tms.k[last], pb, 0, w0, h0, t0, head);
-                  tma_load_5d(dk + kHalfBytes, &tms.k[last], pb, 64, w0, h0, t0, head);
+                  tma_load_5d(dk, &tms.k[last], pb, 0, w0, h0, t0, head_ld);
+                  tma_load_5d(dk + kHalfBytes, &tms.k[last], pb, 64, w0, h0, t0, head_ld);
                 }
                 tile_g = k_tile + 1;
                 ++pair_g;
@@ -703,8 +705,8 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
           const uint32_t pb = bar(kBarPairFull + pair_g % kNumPairBars);
           mbar_expect_tx(pb, (uint32_t)antok * 256u);
           const uint32_t dv = sbase + kOffRing + v_slot * kSlabBytes;
-          tma_load_5d(dv, &tms.v[alast], pb, 0, aw0, ah0, at0, head);
-          tma_load_5d(dv + kHalfBytes, &tms.v[alast], pb, 64, aw0, ah0, at0, head);
+          tma_load_5d(dv, &tms.v[alast], pb, 0, aw0, ah0, at0, head_ld);
+          tma_load_5d(dv + kHalfBytes, &tms.v[alast], pb, 64, aw0, ah0, at0, head_ld);
         }
         ++tile_g;
         ++pair_g;
@@ -1148,7 +1150,7 @@ cudaError_t launch_plan(const HeadParamsArray& hp, const Geom& g, int head0, int
 }
 
 cudaError_t launch_attn(const TensorMaps& tm, const Geom& g, const WorkItem* items, const psa_head_params* hp_dev,
-                        int* ws_header, float* lse, int n_items, int n_sms, cudaStream_t stream) {
+                        int* ws_header, float* lse, int n_items, int n_sms, bool shared_qkv, cudaStream_t stream) {
   {  // per device, cheap: set on every call
     cudaError_t e = cudaFuncSetAttribute(attn_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemAlloc);
     if (e != cudaSuccess) return e;
@@ -1160,6 +1162,7 @@ cudaError_t launch_attn(const TensorMaps& tm, const Geom& g, const WorkItem* ite
   prm.ws_header = ws_header;
   prm.lse = lse;
   prm.n_items = n_items;
+  prm.shared_qkv = shared_qkv ? 1 : 0;
   const int grid = n_items < n_sms ? n_items : n_sms;
   if (grid <= 0) return cudaSuccess;
   attn_fwd_kernel<<<grid, kThreads, kSmemAlloc, stream>>>(tm, prm);

@@ -3,6 +3,7 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <atomic>
 #include <cmath>
 #include <cstring>
@@ -21,7 +22,10 @@ struct TensorMaps {
   CUtensorMap q[2], k[2], v[2], o[2];  // [0]: full 128-token slab box, [1]: a block's last slab
 };
 cudaError_t launch_attn(const TensorMaps& tm, const Geom& g, const WorkItem* items, const psa_head_params* hp_dev,
-                        int* ws_header, float* lse, int n_items, int n_sms, cudaStream_t stream);
+                        int* ws_header, float* lse, int n_items, int n_sms, bool shared_qkv, cudaStream_t stream);
+size_t search_partial_bytes(int n_cand);
+cudaError_t launch_search_losses(const void* outs, const void* ref, long long elems_per_cand, int n_cand, double* partial,
+                                 float* losses, cudaStream_t stream, int* launches);
 cudaError_t launch_wait_probe(int* ws_header, unsigned long long limit_ns, cudaStream_t stream);
 }  // namespace psa
 
@@ -161,13 +165,13 @@ int ensure_workspace(Workspace* w, size_t bytes) {
 }
 
 // `last`: box of a block's last (possibly shorter) slab instead of the full 128-token slab.
-int encode_map(CUtensorMap* tm, const void* base, const Geom& g, const psa_problem* prob, int n_heads_here,
-               bool last = false) {
+int encode_map(CUtensorMap* tm, const void* base, const Geom& g, long long stride_head, long long stride_token,
+               int n_heads_here, bool last) {
   const cuuint64_t dims[5] = {(cuuint64_t)kHeadDim, (cuuint64_t)g.W, (cuuint64_t)g.H, (cuuint64_t)g.T,
                               (cuuint64_t)n_heads_here};
-  const cuuint64_t st = (cuuint64_t)prob->stride_token * 2;
+  const cuuint64_t st = (cuuint64_t)stride_token * 2;
   const cuuint64_t strides[4] = {st, st * g.W, st * g.W * g.H,
-                                 n_heads_here > 1 ? (cuuint64_t)prob->stride_head * 2 : st * g.W * g.H * g.T};
+                                 n_heads_here > 1 ? (cuuint64_t)stride_head * 2 : st * g.W * g.H * g.T};
   cuuint32_t box[5] = {64, (cuuint32_t)g.cw, (cuuint32_t)g.ch, (cuuint32_t)g.ct, 1};
   if (last) box[3 - g.sub_axis] = (cuuint32_t)g.c_last;
   const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
@@ -177,15 +181,23 @@ int encode_map(CUtensorMap* tm, const void* base, const Geom& g, const psa_probl
   return r == CUDA_SUCCESS ? PSA_OK : PSA_ERR_INVALID_ARG;
 }
 
+// Strides (in elements) of the inputs and of the output of one attention launch.
+struct Layout {
+  long long in_head, in_token;    // q, k, v
+  long long out_head, out_token;  // out
+  bool shared_qkv;                // every head reads head 0 of q, k, v
+};
+
 // The four tensors, each with the full-slab box ([0]) and the last-slab box ([1]).
 int encode_maps(TensorMaps* tm, const void* q, const void* k, const void* v, void* out, const Geom& g,
-                const psa_problem* prob, int n_heads_here) {
+                const Layout& lay, int n_heads_here) {
   int rc;
+  const int n_in = lay.shared_qkv ? 1 : n_heads_here;
   for (int last = 0; last < 2; ++last) {
-    if ((rc = encode_map(&tm->q[last], q, g, prob, n_heads_here, last != 0)) != PSA_OK) return rc;
-    if ((rc = encode_map(&tm->k[last], k, g, prob, n_heads_here, last != 0)) != PSA_OK) return rc;
-    if ((rc = encode_map(&tm->v[last], v, g, prob, n_heads_here, last != 0)) != PSA_OK) return rc;
-    if ((rc = encode_map(&tm->o[last], out, g, prob, n_heads_here, last != 0)) != PSA_OK) return rc;
+    if ((rc = encode_map(&tm->q[last], q, g, lay.in_head, lay.in_token, n_in, last != 0)) != PSA_OK) return rc;
+    if ((rc = encode_map(&tm->k[last], k, g, lay.in_head, lay.in_token, n_in, last != 0)) != PSA_OK) return rc;
+    if ((rc = encode_map(&tm->v[last], v, g, lay.in_head, lay.in_token, n_in, last != 0)) != PSA_OK) return rc;
+    if ((rc = encode_map(&tm->o[last], out, g, lay.out_head, lay.out_token, n_heads_here, last != 0)) != PSA_OK) return rc;
   }
   return PSA_OK;
 }
@@ -326,6 +338,52 @@ int psa_mask_build(const psa_head_params* params, const psa_problem* prob, int T
   return PSA_OK;
 }
 
+// Planning + attention launches for n_heads heads (in launches of at most kMaxHeads) on the cached
+// per-device workspace.  Arguments are already validated; g_mu is held by the caller.
+static int run_attn(const void* q, const void* k, const void* v, void* out, float* lse, const psa_head_params* head_params,
+                    int n_heads, const Geom& g, const Layout& lay, cudaStream_t st) {
+  int dev;
+  Workspace* ws;
+  int rc = device_info(&dev, &ws);
+  if (rc != PSA_OK) return rc;
+  if (ws->cc_major != 10) return PSA_ERR_UNSUPPORTED;
+  rc = load_driver_entry();
+  if (rc != PSA_OK) return rc;
+  const int chunk = n_heads < kMaxHeads ? n_heads : kMaxHeads;
+  const size_t items_bytes = sizeof(WorkItem) * (size_t)chunk * g.NB * g.items_per_block;
+  const size_t hp_off = sizeof(int) * kWsHeaderWords;
+  const size_t items_off = (hp_off + sizeof(psa_head_params) * kMaxHeads + 255) & ~size_t(255);
+  rc = ensure_workspace(ws, items_off + items_bytes);
+  if (rc != PSA_OK) return rc;
+  int* ws_header = static_cast<int*>(ws->base);
+  psa_head_params* hp_dev = reinterpret_cast<psa_head_params*>(static_cast<char*>(ws->base) + hp_off);
+  WorkItem* items = reinterpret_cast<WorkItem*>(static_cast<char*>(ws->base) + items_off);
+  for (int head0 = 0; head0 < n_heads; head0 += kMaxHeads) {
+    const int n_here = n_heads - head0 < kMaxHeads ? n_heads - head0 : kMaxHeads;
+    HeadParamsArray hp;
+    std::memset(&hp, 0, sizeof(hp));
+    for (int h = 0; h < n_here; ++h) hp.p[h] = head_params[head0 + h];
+    const long long in_off = lay.shared_qkv ? 0 : (long long)head0 * lay.in_head;
+    const long long out_off = (long long)head0 * lay.out_head;
+    TensorMaps tm;
+    if ((rc = encode_maps(&tm, static_cast<const uint16_t*>(q) + in_off, static_cast<const uint16_t*>(k) + in_off,
+                          static_cast<const uint16_t*>(v) + in_off, static_cast<uint16_t*>(out) + out_off, g, lay, n_here)) != PSA_OK)
+      return rc;
+    Geom gh = g;
+    gh.n_heads = n_here;
+    if (launch_plan(hp, gh, 0, n_here, ws_header, hp_dev, items, st) != cudaSuccess) return PSA_ERR_CUDA;
+    ++g_launches;
+    const int n_items = n_here * g.NB * g.items_per_block;
+    if (g_ev_start && g_ev_stop) cudaEventRecord(g_ev_start, st);
+    if (launch_attn(tm, gh, items, hp_dev, ws_header, lse + (long long)head0 * g.L, n_items, ws->n_sms, lay.shared_qkv, st) !=
+        cudaSuccess)
+      return PSA_ERR_CUDA;
+    if (g_ev_start && g_ev_stop) cudaEventRecord(g_ev_stop, st);
+    ++g_launches;
+  }
+  return PSA_OK;
+}
+
 int psa_attn_fwd(const void* q, const void* k, const void* v, void* out, float* lse, const psa_head_params* head_params,
                  const psa_problem* prob, int T, int H, int W, void* stream) {
   Geom g;
@@ -339,50 +397,73 @@ int psa_attn_fwd(const void* q, const void* k, const void* v, void* out, float* 
   if (prob->n_heads > 1 && (prob->stride_head < kHeadDim || (prob->stride_head % 8) != 0)) return PSA_ERR_INVALID_ARG;
   for (int h = 0; h < prob->n_heads; ++h)
     if (!valid_params(head_params[h])) return PSA_ERR_INVALID_ARG;
-
   std::lock_guard<std::mutex> lock(g_mu);
-  int dev;
-  Workspace* ws;
-  rc = device_info(&dev, &ws);
-  if (rc != PSA_OK) return rc;
-  if (ws->cc_major != 10) return PSA_ERR_UNSUPPORTED;
-  rc = load_driver_entry();
-  if (rc != PSA_OK) return rc;
+  const Layout lay = {prob->stride_head, prob->stride_token, prob->stride_head, prob->stride_token, false};
+  return run_attn(q, k, v, out, lse, head_params, prob->n_heads, g, lay, static_cast<cudaStream_t>(stream));
+}
 
-  const int chunk = prob->n_heads < kMaxHeads ? prob->n_heads : kMaxHeads;
-  const size_t items_bytes = sizeof(WorkItem) * (size_t)chunk * g.NB * g.items_per_block;
-  const size_t hp_off = sizeof(int) * kWsHeaderWords;
-  const size_t items_off = (hp_off + sizeof(psa_head_params) * kMaxHeads + 255) & ~size_t(255);
-  rc = ensure_workspace(ws, items_off + items_bytes);
+int psa_search_select_at_sparsity(const float* losses, const float* sparsity, int n, float target) {
+  if (!losses || !sparsity || n < 1) return PSA_ERR_INVALID_ARG;
+  int best = -1;
+  for (int i = 0; i < n; ++i)
+    if (sparsity[i] >= target && (best < 0 || losses[i] < losses[best])) best = i;
+  return best < 0 ? PSA_ERR_CAPACITY : best;
+}
+
+// ---- PSA-Search for one head (Algorithm 3) ------------------------------------------------------
+// scratch layout: outputs of the n_cand candidates and of full attention ((n_cand + 1) x L x 128 bf16),
+// their lse ((n_cand + 1) x L fp32), the partial sums of the loss reduction.
+static size_t search_out_bytes(int n_cand, long long L) { return ((size_t)(n_cand + 1) * L * kHeadDim * 2 + 255) & ~size_t(255); }
+static size_t search_lse_bytes(int n_cand, long long L) { return ((size_t)(n_cand + 1) * L * 4 + 255) & ~size_t(255); }
+
+int64_t psa_search_scratch_bytes(int n_cand, int T, int H, int W) {
+  if (n_cand < 1 || T < 1 || H < 1 || W < 1) return PSA_ERR_INVALID_ARG;
+  const long long L = (long long)T * H * W;
+  return (int64_t)(search_out_bytes(n_cand, L) + search_lse_bytes(n_cand, L) + search_partial_bytes(n_cand));
+}
+
+int psa_search_losses(const void* q, const void* k, const void* v, const psa_head_params* candidates, int n_cand,
+                      const psa_problem* prob, int T, int H, int W, void* scratch, float* losses, void* stream) {
+  Geom g;
+  int rc = make_geom(prob, T, H, W, true, &g);
   if (rc != PSA_OK) return rc;
-  int* ws_header = static_cast<int*>(ws->base);
-  psa_head_params* hp_dev = reinterpret_cast<psa_head_params*>(static_cast<char*>(ws->base) + hp_off);
-  WorkItem* items = reinterpret_cast<WorkItem*>(static_cast<char*>(ws->base) + items_off);
+  if (!q || !k || !v || !candidates || !scratch || !losses || n_cand < 1) return PSA_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || (reinterpret_cast<uintptr_t>(scratch) & 255u) ||
+      (reinterpret_cast<uintptr_t>(losses) & 3u))
+    return PSA_ERR_INVALID_ARG;
+  if (prob->stride_token < kHeadDim || (prob->stride_token % 8) != 0) return PSA_ERR_INVALID_ARG;
+  // candidate masks, then one all-covering mask: full attention with the same kernel
+  std::vector<psa_head_params> params(candidates, candidates + n_cand);
+  for (int c = 0; c < n_cand; ++c)
+    if (!valid_params(params[c])) return PSA_ERR_INVALID_ARG;
+  const psa_head_params full = {g.Tp, 0, 0, g.Sp, 0, 0};
+  params.push_back(full);
+  char* base = static_cast<char*>(scratch);
+  uint16_t* outs = reinterpret_cast<uint16_t*>(base);
+  float* lse = reinterpret_cast<float*>(base + search_out_bytes(n_cand, g.L));
+  double* partial = reinterpret_cast<double*>(base + search_out_bytes(n_cand, g.L) + search_lse_bytes(n_cand, g.L));
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  std::lock_guard<std::mutex> lock(g_mu);
+  const Layout lay = {0, prob->stride_token, g.L * kHeadDim, kHeadDim, true};
+  rc = run_attn(q, k, v, outs, lse, params.data(), n_cand + 1, g, lay, st);
+  if (rc != PSA_OK) return rc;
+  int launches = 0;
+  const cudaError_t e = launch_search_losses(outs, outs + (long long)n_cand * g.L * kHeadDim, g.L * kHeadDim, n_cand, partial,
+                                             losses, st, &launches);
+  g_launches += launches;
+  return e == cudaSuccess ? PSA_OK : PSA_ERR_CUDA;
+}
 
-  for (int head0 = 0; head0 < prob->n_heads; head0 += kMaxHeads) {
-    const int n_here = prob->n_heads - head0 < kMaxHeads ? prob->n_heads - head0 : kMaxHeads;
-    HeadParamsArray hp;
-    std::memset(&hp, 0, sizeof(hp));
-    for (int h = 0; h < n_here; ++h) hp.p[h] = head_params[head0 + h];
-    const long long eoff = (long long)head0 * prob->stride_head;
-    TensorMaps tm;
-    if ((rc = encode_maps(&tm, static_cast<const uint16_t*>(q) + eoff, static_cast<const uint16_t*>(k) + eoff,
-                          static_cast<const uint16_t*>(v) + eoff, static_cast<uint16_t*>(out) + eoff, g, prob, n_here)) != PSA_OK)
-      return rc;
-    Geom gh = g;
-    gh.n_heads = n_here;
-    if (launch_plan(hp, gh, 0, n_here, ws_header, hp_dev, items, st) != cudaSuccess) return PSA_ERR_CUDA;
-    ++g_launches;
-    const int n_items = n_here * g.NB * g.items_per_block;
-    if (g_ev_start && g_ev_stop) cudaEventRecord(g_ev_start, st);
-    if (launch_attn(tm, gh, items, hp_dev, ws_header, lse + (long long)head0 * g.L, n_items, ws->n_sms, st) !=
-        cudaSuccess)
-      return PSA_ERR_CUDA;
-    if (g_ev_start && g_ev_stop) cudaEventRecord(g_ev_stop, st);
-    ++g_launches;
-  }
-  return PSA_OK;
+int psa_search_select(const float* losses, const float* sparsity, int n, float alpha) {
+  if (!losses || !sparsity || n < 1) return PSA_ERR_INVALID_ARG;
+  // ascending loss, ties by index (stable)
+  std::vector<int> order(n);
+  for (int i = 0; i < n; ++i) order[i] = i;
+  std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return losses[a] < losses[b]; });
+  int best = order[0];
+  for (int i : order)
+    if (losses[i] <= alpha && sparsity[i] > sparsity[best]) best = i;
+  return best;
 }
 
 int psa_attn_fwd_noalloc(const void* q, const void* k, const void* v, void* out, float* lse,
@@ -423,12 +504,13 @@ int psa_attn_fwd_noalloc(const void* q, const void* k, const void* v, void* out,
   std::memset(&hp, 0, sizeof(hp));
   for (int h = 0; h < prob->n_heads; ++h) hp.p[h] = head_params[h];
   TensorMaps tm;
-  if ((rc = encode_maps(&tm, q, k, v, out, g, prob, prob->n_heads)) != PSA_OK) return rc;
+  const Layout lay = {prob->stride_head, prob->stride_token, prob->stride_head, prob->stride_token, false};
+  if ((rc = encode_maps(&tm, q, k, v, out, g, lay, prob->n_heads)) != PSA_OK) return rc;
   // The planning kernel clears the header words (status, ticket) and rewrites the parameter
   // records and every work item of this call, so nothing of the previous call is read.
   if (launch_plan(hp, g, 0, prob->n_heads, header, hp_dev, items, st) != cudaSuccess) return PSA_ERR_CUDA;
   ++g_launches;
-  if (launch_attn(tm, g, items, hp_dev, header, lse, (int)n_items_ll, ws->n_sms, st) != cudaSuccess)
+  if (launch_attn(tm, g, items, hp_dev, header, lse, (int)n_items_ll, ws->n_sms, false, st) != cudaSuccess)
     return PSA_ERR_CUDA;
   ++g_launches;
   if (status_detail) {

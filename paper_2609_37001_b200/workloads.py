@@ -65,3 +65,24 @@ def tensor_bits(seed: int, tensor: str, n_heads: int, L: int, d: int = 128, gain
 def sample_rows(seed: int, head: int, L: int, n: int) -> List[int]:
     gen = np.random.Generator(np.random.Philox(key=(int(seed) << 20) ^ (7 << 16) ^ int(head)))
     return sorted(set(int(x) for x in gen.integers(0, L, size=n)))
+
+
+def search_candidates(seed: int, n: int, grid: Sequence[int], tile: Sequence[int]) -> List[Tuple[int, ...]]:
+    """n distinct seeded candidate masks (Tw, To, Ts, Sw, So, Ss) from the initialisation space the
+    paper gives for PSA-Search: 0 < Tw < T/bt, To in {0, +-1, +-2}, Ts in {1, 2, 3, inf},
+    0 < Sw < W/bw, So in {0, +-1}, Ss in {1, 3, 5, 6, inf} (inf is encoded as stride 0).  Widths are
+    clamped to at least 1 on tiny grids; fewer than n are returned if the space is smaller."""
+    T, H, W = (int(x) for x in grid)
+    tw_hi = max(2, -(-T // int(tile[0])))
+    sw_hi = max(2, -(-W // int(tile[2])))
+    gen = np.random.Generator(np.random.Philox(key=(int(seed) << 20) ^ (9 << 16)))
+    seen, out = set(), []
+    for _ in range(200 * n):
+        c = (int(gen.integers(1, tw_hi)), int(gen.choice([0, 1, -1, 2, -2])), int(gen.choice([1, 2, 3, 0])),
+             int(gen.integers(1, sw_hi)), int(gen.choice([0, 1, -1])), int(gen.choice([1, 3, 5, 6, 0])))
+        if c not in seen:
+            seen.add(c)
+            out.append(c)
+            if len(out) == n:
+                break
+    return out

@@ -72,3 +72,37 @@ def test_losses_against_direct_formulas():
         want = float(((out - full) ** 2).sum() / (L * d))
         assert abs(losses[c] - want) < 1e-14
     assert 0 < losses[1] < losses[2]             # dropping more keys moves the output further
+
+
+def test_select_at_sparsity_is_min_loss_over_the_feasible_set():
+    assert O.search_select_at_sparsity([0.02, 0.001, 0.008, 0.004], [0.9, 0.1, 0.75, 0.5], 0.5) == 3
+    assert O.search_select_at_sparsity([0.02, 0.001, 0.008, 0.004], [0.9, 0.1, 0.75, 0.5], 0.8) == 0
+    assert O.search_select_at_sparsity([0.02, 0.001], [0.9, 0.1], 0.95) == -1
+    assert O.search_select_at_sparsity([0.5, 0.5], [0.6, 0.7], 0.6) == 0      # tie: lower index
+    rng = random.Random(8)
+    for _ in range(300):
+        n = rng.randint(1, 9)
+        losses = [rng.randint(0, 20) / 20 for _ in range(n)]
+        spars = [rng.choice([0.1, 0.25, 0.5, 0.75, 0.9]) for _ in range(n)]
+        target = rng.random()
+        got = O.search_select_at_sparsity(losses, spars, target)
+        ok = [i for i in range(n) if spars[i] >= target]
+        if not ok:
+            assert got == -1
+        else:
+            # brute force over every feasible candidate
+            assert got in ok and all(losses[got] <= losses[i] for i in ok)
+            assert got == min(i for i in ok if losses[i] == losses[got])
+
+
+def test_the_two_interfaces_agree_on_the_pareto_front():
+    # choosing by threshold alpha and then asking for that candidate's sparsity returns a candidate
+    # of no larger loss and no smaller sparsity
+    rng = random.Random(10)
+    for _ in range(200):
+        n = rng.randint(2, 9)
+        losses = [rng.randint(0, 50) / 50 for _ in range(n)]
+        spars = [rng.choice([0.1, 0.25, 0.5, 0.75, 0.9]) for _ in range(n)]
+        a = O.search_select(losses, spars, rng.random())
+        b = O.search_select_at_sparsity(losses, spars, spars[a])
+        assert b >= 0 and losses[b] <= losses[a] and spars[b] >= spars[a]

@@ -1,0 +1,135 @@
+"""PSA-Search inner loop (Algorithm 3) through the C ABI against the fp64 oracle.
+
+psa_search_losses: the CUDA path computes every candidate's output and full attention's with the
+stripe attention kernel (bf16 outputs) and reduces the mean squared difference on the device; the
+oracle does the same in fp64 from the definition.  Tolerance: both outputs carry an error of at
+most e = 2^-8 * rms(full output) (bf16 rounding of the output, of the probabilities and of the
+accumulation order), so the difference d' = d + err obeys
+|mean(d'^2) - mean(d^2)| <= 2*sqrt(loss)*(2e) + (2e)^2.
+psa_search_select is integer/compare work: the chosen index must be identical."""
+import math
+import random
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import psa_oracle as O
+from paper_2609_37001_b200 import workloads as WL
+
+INF = O.INF_STRIDE
+SCALE = 1.0 / math.sqrt(128.0)
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2609_37001_b200 import build
+    build.build()
+    from paper_2609_37001_b200 import binding
+    return binding
+
+
+def _to_dev(bits):
+    return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+
+
+def _sparsities(cands, grid, tile):
+    return [O.tile_sparsity(tuple(p), *grid, tuple(tile)) for p in cands]
+
+
+def _check_losses(B, cands, grid, tile, seed, gain):
+    T, H, W = grid
+    L = T * H * W
+    bits = {n: WL.head_bits(seed, n, 0, L, gain=(gain if n != "v" else 1.0)) for n in ("q", "k", "v")}
+    q, k, v = (_to_dev(bits[n]) for n in ("q", "k", "v"))
+    got = B.psa_search_losses(q, k, v, cands, grid, tile, SCALE).cpu().numpy().astype(np.float64)
+    st, detail = B.psa_last_device_status()
+    assert st == 0, (st, hex(detail))
+    qf, kf, vf = (O.bf16_bits_to_f64(bits[n]) for n in ("q", "k", "v"))
+    ref = O.search_losses(qf, kf, vf, [tuple(p) for p in cands], T, H, W, tuple(tile), SCALE)
+    full, _ = O.dense_attention(qf, kf, vf, SCALE)
+    e2 = 2.0 * 2.0 ** -8 * math.sqrt(np.mean(full ** 2))
+    tol = 2.0 * np.sqrt(ref) * e2 + e2 * e2
+    assert np.all(np.abs(got - ref) <= tol), (got, ref, tol)
+    return got, ref
+
+
+@pytest.mark.gpu
+def test_losses_ragged_grid_single_slab_blocks(B):
+    grid, tile = (5, 20, 24), (1, 8, 16)
+    Tp, Hp, Wp = O.block_grid(*grid, tile)
+    Sp = Hp * Wp
+    cands = [(Tp, 0, INF, Sp, 0, INF),   # all-covering: loss 0 up to output rounding
+             (1, 0, INF, Sp, 0, INF),    # own frame only
+             (2, 0, INF, 2, 0, INF),
+             (1, 0, 2, 1, 0, 3),         # strided in both axes
+             (1, 1, INF, Sp, 0, INF),    # neighbouring frames only: never the own frame
+             (1, Tp, INF, 1, 0, INF),    # offset beyond the grid: every row empty, out = 0
+             (Tp, 0, INF, 1, 0, 2)]
+    got, ref = _check_losses(B, cands, grid, tile, seed=31, gain=3.0)
+    assert got[0] <= (2.0 ** -8) ** 2 * 4
+    # the all-empty candidate's loss is the mean square of full attention's output
+    assert abs(got[5] - ref[5]) <= 1e-2 * ref[5]
+    # the selection on the device losses equals the selection on the oracle's
+    sp = _sparsities(cands, grid, tile)
+    for alpha in (0.0, float(np.median(ref)), float(ref.max()) * 2):
+        assert B.psa_search_select(list(got), sp, alpha) == O.search_select(list(got.astype(np.float32)), sp, np.float32(alpha))
+
+
+@pytest.mark.gpu
+def test_losses_two_slab_blocks(B):
+    grid, tile = (3, 30, 32), (1, 15, 16)
+    Tp, Hp, Wp = O.block_grid(*grid, tile)
+    Sp = Hp * Wp
+    cands = [(1, 0, INF, Sp, 0, INF), (Tp, 0, INF, 1, 0, INF), (1, 0, 2, 2, 0, INF), (2, -1, INF, 1, 1, 2)]
+    _check_losses(B, cands, grid, tile, seed=32, gain=2.0)
+
+
+@pytest.mark.gpu
+def test_losses_more_candidates_than_one_launch_holds(B):
+    # 150 candidates + full attention: two launches of the attention kernel over one scratch buffer
+    grid, tile = (3, 8, 32), (1, 8, 16)
+    Tp, Hp, Wp = O.block_grid(*grid, tile)
+    Sp = Hp * Wp
+    rng = random.Random(5)
+    base = [(rng.randint(1, Tp), rng.randint(-1, 1), rng.choice([INF, 2, 3]),
+             rng.randint(1, Sp), rng.randint(-1, 1), rng.choice([INF, 2])) for _ in range(10)]
+    cands = [base[i % 10] for i in range(150)]
+    got, ref = _check_losses(B, cands, grid, tile, seed=33, gain=2.0)
+    # equal candidates give bit-equal losses wherever they sit in the batch
+    for i in range(150):
+        assert got[i] == got[i % 10]
+
+
+@pytest.mark.gpu
+def test_search_rejects_bad_arguments(B):
+    q = torch.zeros(256, 128, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(RuntimeError):
+        B.psa_search_losses(q, q, q, [(0, 0, 0, 1, 0, 0)], (1, 16, 16), (1, 8, 16), SCALE)   # width 0
+    with pytest.raises(ValueError):
+        B.psa_search_losses(q, q, q, [(1, 0, 0, 1, 0, 0)], (1, 16, 16), (1, 8, 16), SCALE,
+                            scratch=torch.empty(256, dtype=torch.uint8, device="cuda"))
+    assert B.psa_last_device_status()[0] == 0
+
+
+def test_select_matches_oracle_and_hand_examples(B):
+    # host-only entry point: runs without a GPU
+    losses = [0.020, 0.001, 0.008, 0.004]
+    spars = [0.90, 0.10, 0.75, 0.50]
+    assert B.psa_search_select(losses, spars, 0.0005) == 1
+    assert B.psa_search_select(losses, spars, 0.005) == 3
+    assert B.psa_search_select(losses, spars, 0.01) == 2
+    assert B.psa_search_select(losses, spars, 0.05) == 0
+    assert B.psa_search_select([0.25, 0.125, 0.375], [0.5, 0.5, 0.5], 1.0) == 1
+    assert B.psa_search_select([0.25, 0.125], [0.875, 0.25], 0.25) == 0
+    rng = random.Random(9)
+    for _ in range(500):
+        n = rng.randint(1, 12)
+        ls = [rng.randint(0, 64) / 64.0 for _ in range(n)]          # exact in fp32, many ties
+        sp = [rng.choice([0.125, 0.25, 0.5, 0.75, 0.875]) for _ in range(n)]
+        alpha = rng.randint(0, 64) / 64.0
+        assert B.psa_search_select(ls, sp, alpha) == O.search_select(ls, sp, alpha)
+        target = rng.randint(0, 8) / 8.0
+        assert B.psa_search_select_at_sparsity(ls, sp, target) == O.search_select_at_sparsity(ls, sp, target)
+    with pytest.raises(ValueError):
+        B.psa_search_select([0.1], [0.1, 0.2], 0.5)
