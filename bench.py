@@ -418,6 +418,105 @@ def run_report(args):
     sys.stderr.write(text)
 
 
+def run_search(args, w):
+    """PSA-Search inner loop (Algorithm 3) for ONE head of the workload's shape: psa_search_losses over
+    N seeded candidates drawn from the paper's initialisation space, then psa_search_select.  Prints one
+    JSON line: candidates per second, the tensor roofline of the attention launch inside it, the HBM
+    roofline of the loss reduction, and the oracle timed on sampled query rows."""
+    import torch
+    from paper_2609_37001_b200 import build
+    build.build()
+    from paper_2609_37001_b200 import binding as B
+    from paper_2609_37001_b200 import workloads as WL
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    peaks = load_peaks()
+    T, H, W = w["grid"]
+    L, tile = T * H * W, w["tile"]
+    cands = WL.search_candidates(w["seed"], args.search, w["grid"], tile)
+    n = len(cands)
+    bits = {t: WL.head_bits(w["seed"], t, 0, L) for t in ("q", "k", "v")}
+    q, k, v = (torch.from_numpy(bits[t].view(np.int16)).view(torch.bfloat16).to(dev) for t in ("q", "k", "v"))
+    scratch = torch.empty(B.psa_search_scratch_bytes(n, w["grid"]), dtype=torch.uint8, device=dev)
+    # attended real (query, key) pairs of every candidate from the library's own block masks
+    Tp, Hp, Wp = -(-T // tile[0]), -(-H // tile[1]), -(-W // tile[2])
+    real = lambda n_tok, b, nb_: torch.tensor([min(b, n_tok - i * b) for i in range(nb_)], dtype=torch.float64)
+    rt, rh, rw = real(T, tile[0], Tp), real(H, tile[1], Hp), real(W, tile[2], Wp)
+    real_blk = (rt[:, None, None] * rh[None, :, None] * rw[None, None, :]).reshape(-1).to(dev)
+    pairs, spars = [], []
+    for c0 in range(0, n, 16):
+        m, _, _ = B.psa_mask_build(cands[c0:c0 + 16], w["grid"], tile)
+        md = m.to(torch.float64)
+        pairs += [float(x) for x in torch.einsum("hqk,q,k->h", md, real_blk, real_blk).cpu()]
+        spars += [float(x) for x in (1.0 - md.mean(dim=(1, 2))).cpu()]
+        del m, md
+    flops = 4.0 * HEAD_DIM * (sum(pairs) + float(L) * L)
+    stream = torch.cuda.Stream(device=dev)
+    with torch.cuda.stream(stream):
+        for _ in range(max(args.warmup, 3)):
+            losses = B.psa_search_losses(q, k, v, cands, w["grid"], tile, SCALE, scratch=scratch, stream=stream)
+        kev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+        for a, b in kev:
+            a.record(stream); b.record(stream)
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        sampler = ClockSampler(0)
+        torch.cuda.synchronize()
+        launches0 = B.psa_launch_count()
+        ev0.record(stream)
+        for i in range(args.steps):
+            B.psa_profile_events(*kev[i])
+            losses = B.psa_search_losses(q, k, v, cands, w["grid"], tile, SCALE, scratch=scratch, stream=stream)
+        ev1.record(stream)
+        torch.cuda.synchronize()
+        launches = B.psa_launch_count() - launches0
+        B.psa_profile_events(None, None)
+        clocks = sampler.stop()
+        st, detail = B.psa_last_device_status()
+        if st != 0:
+            raise SystemExit(f"device status {st} detail {hex(detail)}")
+    ms = ev0.elapsed_time(ev1) / args.steps
+    attn_ms = float(np.mean([a.elapsed_time(b) for a, b in kev]))  # the (last) attention launch of each call
+    lh = losses.cpu().tolist()
+    alpha = float(np.median(lh))
+    chosen = B.psa_search_select(lh, spars, alpha)
+    loss_bytes = (n + 1) * L * HEAD_DIM * 2   # every candidate output once + the reference once
+    line = {"metric": "psa_search_candidates_per_s", "value": n / (ms * 1e-3), "unit": "candidates/s", "n_gpus": 1,
+            "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": w["name"] + "_search_1head", "grid": w["grid"], "tokens": L, "mask_block": tile,
+                       "n_candidates": n, "mean_candidate_tile_sparsity": float(np.mean(spars)),
+                       "step": "psa_search_losses (plan + attention over candidates and full attention + loss reduction)"},
+            "roofline": {"bound": "tensor", "kernel": "attn_fwd_kernel", "achieved": flops / (attn_ms * 1e-3) / 1e12,
+                         "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                         "frac": flops / (attn_ms * 1e-3) / 1e12 / peaks["bf16_tflops"], "kernel_ms": attn_ms,
+                         "algorithmic_flops_per_launch": flops, "traffic": None,
+                         "note": "valid when candidates + 1 <= 128 (one attention launch per call)"},
+            "loss_reduction": {"ms": ms - attn_ms, "bytes": loss_bytes, "GBps": loss_bytes / ((ms - attn_ms) * 1e-3) / 1e9,
+                               "hbm_peak_GBps": peaks["hbm_gbs"], "note": "step time minus the attention launch: plan + two reduction kernels"},
+            "selection": {"alpha": alpha, "chosen": int(chosen), "chosen_params": list(cands[chosen]),
+                          "chosen_sparsity": spars[chosen], "chosen_loss": lh[chosen]},
+            "clocks": clocks, "gpu_launches": int(launches)}
+    if not args.quick:
+        from oracle import psa_oracle as O
+        qf, kf, vf = (O.bf16_bits_to_f64(bits[t]) for t in ("q", "k", "v"))
+        rows = WL.sample_rows(w["seed"], 0, L, 16)
+        t0, done = time.perf_counter(), 0
+        O.attention_rows(qf, kf, vf, rows, (Tp, 0, 0, Hp * Wp, 0, 0), T, H, W, tuple(tile), SCALE)
+        for c in cands:
+            O.attention_rows(qf, kf, vf, rows, tuple(c), T, H, W, tuple(tile), SCALE)
+            done += 1
+            if time.perf_counter() - t0 > 15.0:
+                break
+        secs = time.perf_counter() - t0
+        line["cpu_baseline"] = {"value": done / (secs * L / len(rows)), "unit": "candidates/s", "cores": blas_threads(),
+                                "kind": "oracle", "seconds": secs,
+                                "sample": f"{done} candidates + full attention on {len(rows)} seeded query rows each, "
+                                          f"scaled by {L}/{len(rows)} rows"}
+    print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -428,7 +527,13 @@ def main():
     ap.add_argument("--quick", action="store_true", help="timed region only (no dense/e2e/CPU legs); for profiling")
     ap.add_argument("--report", default=None, metavar="FILE.md",
                     help="time every workload (PSA, dense, mask build) on one GPU and write a markdown table; no JSON line")
+    ap.add_argument("--search", type=int, default=0, metavar="N",
+                    help="time the PSA-Search inner loop for one head over N seeded candidates instead of the hot path")
     args = ap.parse_args()
+    if args.search:
+        from paper_2609_37001_b200 import workloads as WL
+        run_search(args, WL.workload(args.workload))
+        return
     if args.report:
         run_report(args)
         return
