@@ -20,7 +20,7 @@
 // P_i overwrite the first columns of S_i.  A key slab has 128 keys, or 112/96/64 for the last
 // slab of a block whose token count is not a multiple of 128.
 // Every wait is bounded; on expiry the CTA records a status word and unwinds.
-// Build-time knobs: PSA_SPLIT_P (publish P in two halves, default 1), PSA_EMU_PAIRS (share of
+// Build-time knobs: PSA_EMU_PAIRS (share of
 // exponentials computed by a polynomial on the FMA pipe, default 0), PSA_TRACE (cycle stamps).
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -30,6 +30,11 @@
 namespace psa {
 
 constexpr int kThreads = 384;                       // 3 warpgroups; register budgets are re-split below
+#if !defined(PSA_UTIL_FIRST) || PSA_UTIL_FIRST
+constexpr int kWarpMma = 0, kWarpLoad = 1, kUtilGroup = 0, kFirstSoftmaxWarp = 4;
+#else
+constexpr int kWarpMma = 9, kWarpLoad = 8, kUtilGroup = 2, kFirstSoftmaxWarp = 0;
+#endif
 constexpr int kNumSlots = 5;                       // K/V ring slots of one 128 x 128 bf16 slab
 constexpr uint32_t kSlabBytes = 128 * 128 * 2;     // 32 KB
 constexpr uint32_t kHalfBytes = kSlabBytes / 2;    // one 64-column swizzled half
@@ -53,7 +58,7 @@ constexpr uint32_t kOffSched = kOffMaskS + (kMaxSp / 32) * 4;   // two published
 constexpr uint32_t kOffMisc = kOffSched + 32;                   // tmem base, abort flag
 constexpr uint32_t kOffXchg = kOffMisc + 16;                    // split-KV merge: (m, l) of 128 rows
 constexpr uint32_t kSmemBytes = kOffXchg + 128 * 8;
-constexpr uint32_t kSmemAlloc = kSmemBytes + 1024;              // slack for manual alignment
+constexpr uint32_t kSmemAlloc = kSmemBytes;                     // base alignment comes from the declaration
 static_assert(kSmemAlloc <= 232448, "exceeds the 227 KB of shared memory a CTA may use");
 
 // ----------------------------------------------------------------------------- PTX
@@ -103,6 +108,42 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 // warp-uniform variant: every lane waits, the warp agrees on the outcome
 __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag, int code) {
   const bool ok = mbar_wait(bar, parity, abort_flag, code);
+  return __all_sync(0xffffffffu, ok);
+}
+
+// Two barriers at once: both probes are issued before either result is used, so a wait that is
+// already satisfied costs one shared-memory round trip instead of two.
+__device__ __forceinline__ bool mbar_wait2_warp(uint32_t bar_a, uint32_t par_a, uint32_t bar_b, uint32_t par_b,
+                                                volatile int* abort_flag, int code_a, int code_b) {
+  uint32_t ra, rb;
+  asm volatile(
+      "{\n\t.reg .pred pa, pb;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 pa, [%2], %3;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 pb, [%4], %5;\n\t"
+      "selp.u32 %0, 1, 0, pa;\n\t"
+      "selp.u32 %1, 1, 0, pb;\n\t}"
+      : "=r"(ra), "=r"(rb) : "r"(bar_a), "r"(par_a), "r"(bar_b), "r"(par_b) : "memory");
+  bool ok = true;
+  if (!ra) ok = mbar_wait(bar_a, par_a, abort_flag, code_a);
+  if (ok && !rb) ok = mbar_wait(bar_b, par_b, abort_flag, code_b);
+  return __all_sync(0xffffffffu, ok);
+}
+
+// Waits on barrier a and, in the same shared-memory round trip, probes barrier b once;
+// *b_done tells whether b's phase was already complete (warp-uniform).
+__device__ __forceinline__ bool mbar_wait_probe_warp(uint32_t bar_a, uint32_t par_a, uint32_t bar_b, uint32_t par_b,
+                                                     volatile int* abort_flag, int code_a, bool* b_done) {
+  uint32_t ra, rb;
+  asm volatile(
+      "{\n\t.reg .pred pa, pb;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 pa, [%2], %3;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 pb, [%4], %5;\n\t"
+      "selp.u32 %0, 1, 0, pa;\n\t"
+      "selp.u32 %1, 1, 0, pb;\n\t}"
+      : "=r"(ra), "=r"(rb) : "r"(bar_a), "r"(par_a), "r"(bar_b), "r"(par_b) : "memory");
+  bool ok = true;
+  if (!ra) ok = mbar_wait(bar_a, par_a, abort_flag, code_a);
+  *b_done = __all_sync(0xffffffffu, rb != 0u);
   return __all_sync(0xffffffffu, ok);
 }
 
@@ -243,8 +284,8 @@ __device__ __forceinline__ void exp2_poly_pair(uint64_t x2, float& p0, float& p1
 #ifndef PSA_EMU_PAIRS
 #define PSA_EMU_PAIRS 0   // of every 4 pairs of probabilities, this many use exp2_poly_pair (0: all ex2.approx)
 #endif
-#ifndef PSA_SPLIT_P
-#define PSA_SPLIT_P 1     // publish P in two halves of 64 keys
+#ifndef PSA_UTIL_FIRST
+#define PSA_UTIL_FIRST 1  // 1: MMA and load warps are warps 0 and 1 (oldest warps of their schedulers); 0: warps 9 and 8
 #endif
 
 
@@ -271,10 +312,11 @@ __device__ __forceinline__ bool elect_one() {
 #ifdef PSA_TRACE
 __device__ long long g_trace[4 * 64 * 8];
 __device__ long long g_trace_items[2 * 256 * 4];
+__device__ long long g_trace_w[8 * 64 * 2];
 #define TRACE(role, j, k)                                                                     \
   do {                                                                                          \
     if (blockIdx.x == 0 && n == 1 && (j) < 64 && (threadIdx.x & 31) == 0 &&                     \
-        ((threadIdx.x >> 5) & 3) == ((role) < 2 ? 0 : 1))                                       \
+        ((threadIdx.x >> 5) & 3) == (((role) < 2 ? kFirstSoftmaxWarp : kWarpMma) & 3))         \
       g_trace[((role) * 64 + (j)) * 8 + (k)] = clock64();                                       \
   } while (0)
 #else
@@ -465,7 +507,6 @@ __device__ __forceinline__ void softmax_slab(uint32_t tS, uint32_t tO, const uin
     uint32_t pk[16];
     exp_chunk(c4 * 32, 16, pk);
     tc_st16(tS + c4 * 16, pk);
-#if PSA_SPLIT_P
     if (c4 == 1) {  // the first 64 keys are final: their P V MMAs may start
       STAMP(5);
       tc_wait_st();
@@ -473,7 +514,6 @@ __device__ __forceinline__ void softmax_slab(uint32_t tS, uint32_t tO, const uin
       mbar_arrive(bar_half);
       STAMP(3);
     }
-#endif
   }
   if (REM) {
     uint32_t pk[16];
@@ -492,8 +532,10 @@ __device__ __forceinline__ void softmax_slab(uint32_t tS, uint32_t tO, const uin
 
 __global__ void __launch_bounds__(kThreads, 1)
 attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  // 128-byte swizzled slabs need a 1024-byte aligned base; the declaration asks for it and the
+  // kernel checks it (a misaligned base is reported through the status word, no work is done).
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  uint8_t* smem = smem_raw;
   const uint32_t sbase = smem_u32(smem);
   const Geom& g = prm.g;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -527,7 +569,7 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
     for (int s = 0; s < kNumSlots; ++s) mbar_init(bar(kBarSlotEmpty + s), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 9) {
+  if (warp == kWarpMma) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(sbase + kOffMisc), "r"(512) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -538,8 +580,8 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
   // the constant keeps every TMEM address of the MMA stream in uniform registers.  Checked:
   // any other base is reported through the status word and the CTA does no work.
   constexpr uint32_t tmem = 0u;
-  const bool tmem_ok = (*tmem_slot == 0u);
-  if (!tmem_ok && threadIdx.x == 0) atomicCAS((int*)abort_flag, 0, 0x500);
+  const bool tmem_ok = (*tmem_slot == 0u) && ((sbase & 1023u) == 0u);
+  if (!tmem_ok && threadIdx.x == 0) atomicCAS((int*)abort_flag, 0, (*tmem_slot == 0u) ? 0x501 : 0x500);
 
   // Work items are handed out through a two-entry ring: the load warp draws a ticket from
   // a global counter (items are stored heaviest first), publishes the item, and the other
@@ -559,10 +601,10 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
     return wi.x >= 0;
   };
 
-  if (warp >= 8) {
+  if ((warp >> 2) == kUtilGroup) {
   // Third warpgroup: give registers away (the budget is re-split per warpgroup).
   asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
-  if (warp == 8) {
+  if (warp == kWarpLoad) {
     // ======================================================================= load warp
     // Ring tiles are issued in the order K_0, V_0, K_1, V_1, ...; the MMA warp needs V_j and
     // K_{j+1} at the same moment, so those two travel under one "pair" barrier
@@ -737,7 +779,7 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
       }
     }
     __syncwarp();
-  } else if (warp == 9) {
+  } else if (warp == kWarpMma) {
     // ======================================================================= MMA warp
     constexpr uint32_t kIdescPV = instr_desc(true, 128);  // N = head_dim
     uint32_t tile_g = 0, pair_g = 0;
@@ -777,7 +819,10 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
     };
 
     uint32_t it_o0 = 0, it_o1 = 0;    // items in which accumulator O_i was used
-    auto nk_of = [&](int j) -> int { return (j % g.n_sub == g.n_sub - 1) ? g.n_last : kSlabTokens; };
+    // keys of a slab from its index within its block (r = j mod n_sub, carried along: no division)
+    const int r_last = g.n_sub - 1;
+    auto nk_at = [&](int r) -> int { return r == r_last ? g.n_last : kSlabTokens; };
+    auto r_inc = [&](int r) -> int { return r == r_last ? 0 : r + 1; };
 
     for (uint32_t n = 0; ok; ++n) {
       WorkItem wi;
@@ -812,6 +857,7 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
       if (n_kv > 0 && split) {
         // ---- split-KV item: one query slab (Q buffer 0); key slab j feeds tile (j & 1).
         // Ring order (see the load warp): K_0, K_1, (V_0, K_2), (V_1, K_3), ..., V_{n-2}, V_{n-1}.
+        int r0 = 0;   // residue of the slab whose scores are issued next
         for (int j = 0; ok && j < 2 && j < n_kv; ++j) {
           ok = mbar_wait_warp(bar(kBarPairFull + pair_g % kNumPairBars), (pair_g / kNumPairBars) & 1u, abort_flag, 0x230);
           if (!ok) break;
@@ -820,12 +866,14 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
           ++tile_g;
           tc_fence_after();
           if (elect_one()) {
-            issue_qk(0, slot, nk_of(j), j);
+            issue_qk(0, slot, nk_at(r0), j);
             tc_commit(bar(kBarSFull + j));
             tc_commit(bar(kBarSlotEmpty + slot));
           }
           __syncwarp();
+          r0 = r_inc(r0);
         }
+        int rj = 0;   // residue of slab j; r0 is that of slab j + 2 from here on
         for (int j = 0; ok && j < n_kv; ++j) {
           const int i = j & 1;
           ok = mbar_wait_warp(bar(kBarPairFull + pair_g % kNumPairBars), (pair_g / kNumPairBars) & 1u, abort_flag, 0x231);
@@ -836,27 +884,22 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
           const uint32_t kslot = (tile_g + 1) % kNumSlots;
           tile_g += more ? 2u : 1u;
           const uint32_t cs = i == 0 ? cnt_s0 : cnt_s1;
-          const int nk_cur = nk_of(j);
-#if PSA_SPLIT_P
+          const int nk_cur = nk_at(rj);
+          rj = r_inc(rj);
           ok = mbar_wait_warp(bar(kBarPHalf + i), cs & 1u, abort_flag, 0x234 + i);
           if (!ok) break;
           tc_fence_after();
           if (elect_one()) issue_pv_half(i, vslot, 0, j > 1, nk_cur);
-#endif
           ok = mbar_wait_warp(bar(kBarPReady + i), cs & 1u, abort_flag, 0x232 + i);
           if (!ok) break;
           if (i == 0) ++cnt_s0; else ++cnt_s1;
           tc_fence_after();
           if (elect_one()) {
-#if PSA_SPLIT_P
             issue_pv_half(i, vslot, 1, true, nk_cur);
-#else
-            issue_pv_half(i, vslot, 0, j > 1, nk_cur);
-            issue_pv_half(i, vslot, 1, true, nk_cur);
-#endif
             tc_commit(bar(kBarSlotEmpty + vslot));
             if (more) {
-              issue_qk(0, kslot, nk_of(j + 2), i);
+              issue_qk(0, kslot, nk_at(r0), i);
+              r0 = r_inc(r0);
               tc_commit(bar(kBarSFull + i));
               tc_commit(bar(kBarSlotEmpty + kslot));
             } else {
@@ -879,7 +922,7 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
 #pragma unroll
             for (int i = 0; i < 2; ++i) {
               if (i < nq) {
-                issue_qk(i, slot, nk_of(0), i);
+                issue_qk(i, slot, nk_at(0), i);
                 tc_commit(bar(kBarSFull + i));
               }
             }
@@ -887,42 +930,47 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
           }
           __syncwarp();
         }
+        int rj = 0;
         for (int j = 0; ok && j < n_kv; ++j) {
-          const int nk_cur = nk_of(j);
-          const int nk_next = nk_of(j + 1);
-          // V_j and (unless this is the last slab) K_{j+1} arrive under one barrier
+          const int nk_cur = nk_at(rj);
+          rj = r_inc(rj);
+          const int nk_next = nk_at(rj);
+          // V_j and (unless this is the last slab) K_{j+1} arrive under one barrier; it is waited
+          // for together with the first half of P_0 (one shared-memory round trip for both)
           TRACE(2, j, 5);
-          ok = mbar_wait_warp(bar(kBarPairFull + pair_g % kNumPairBars), (pair_g / kNumPairBars) & 1u, abort_flag, 0x211);
-          if (!ok) break;
-          TRACE(2, j, 3);
-          ++pair_g;
           const bool more = (j + 1 < n_kv);
           const uint32_t vslot = tile_g % kNumSlots;
           const uint32_t kslot = (tile_g + 1) % kNumSlots;
           tile_g += more ? 2u : 1u;
+          ok = mbar_wait2_warp(bar(kBarPairFull + pair_g % kNumPairBars), (pair_g / kNumPairBars) & 1u,
+                               bar(kBarPHalf + 0), cnt_s0 & 1u, abort_flag, 0x211, 0x224);
+          if (!ok) break;
+          TRACE(2, j, 3);
+          ++pair_g;
+          bool half1_done = false;   // first half of P_1 already seen complete
 #pragma unroll
           for (int i = 0; i < 2; ++i) {
             if (!ok || i >= nq) break;
             const uint32_t cs = i == 0 ? cnt_s0 : cnt_s1;
-#if PSA_SPLIT_P
-            ok = mbar_wait_warp(bar(kBarPHalf + i), cs & 1u, abort_flag, 0x224 + i);
-            if (!ok) break;
+            if (i == 1 && !half1_done) {
+              ok = mbar_wait_warp(bar(kBarPHalf + 1), cs & 1u, abort_flag, 0x225);
+              if (!ok) break;
+            }
             tc_fence_after();
             TRACE(2 + i, j, 0);
             if (elect_one()) issue_pv_half(i, vslot, 0, j > 0, nk_cur);
-#endif
-            ok = mbar_wait_warp(bar(kBarPReady + i), cs & 1u, abort_flag, 0x220 + i);
+            if (i == 0 && nq > 1) {
+              ok = mbar_wait_probe_warp(bar(kBarPReady + 0), cs & 1u, bar(kBarPHalf + 1), cnt_s1 & 1u, abort_flag,
+                                        0x220, &half1_done);
+            } else {
+              ok = mbar_wait_warp(bar(kBarPReady + i), cs & 1u, abort_flag, 0x220 + i);
+            }
             if (!ok) break;
             if (i == 0) ++cnt_s0; else ++cnt_s1;
             tc_fence_after();
             TRACE(2 + i, j, 1);
             if (elect_one()) {
-#if PSA_SPLIT_P
               issue_pv_half(i, vslot, 1, true, nk_cur);
-#else
-              issue_pv_half(i, vslot, 0, j > 0, nk_cur);
-              issue_pv_half(i, vslot, 1, true, nk_cur);
-#endif
               if (i == nq - 1) tc_commit(bar(kBarSlotEmpty + vslot));
               if (more) {
                 issue_qk(i, kslot, nk_next, i);
@@ -953,7 +1001,7 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
   } else {
     asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
     // ======================================================================= softmax warps
-    const int qi = warp >> 2;                     // tile (S_i, O_i) handled by this warpgroup
+    const int qi = (warp - kFirstSoftmaxWarp) >> 2;   // tile (S_i, O_i) handled by this warpgroup
     const int row = (warp & 3) * 32 + lane;       // row of the slab == TMEM lane
     const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
     const uint32_t tS = tmem + lane_addr + (uint32_t)qi * 128u;
@@ -976,8 +1024,12 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
       if (active) {
         // key slabs of this tile: all of them, or every second one in a split-KV item
         const int j0 = split ? qi : 0, dj = split ? 2 : 1;
+        const int r_last = g.n_sub - 1;
+        int rj = (j0 > r_last) ? 0 : j0;   // j mod n_sub, carried along (no division in the loop)
         for (int j = j0; ok && j < n_kv; j += dj) {
-          const int nk = (j % g.n_sub == g.n_sub - 1) ? g.n_last : kSlabTokens;
+          const int nk = (rj == r_last) ? g.n_last : kSlabTokens;
+          rj = (rj == r_last) ? 0 : rj + 1;
+          if (dj == 2) rj = (rj == r_last) ? 0 : rj + 1;
           ok = mbar_wait_warp(bar(kBarSFull + qi), cnt_s & 1u, abort_flag, 0x300 + qi);
           if (!ok) break;
           ++cnt_s;
@@ -993,11 +1045,17 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
           long long* tr = nullptr;
 #endif
           const bool first = (j == j0);
+#ifdef PSA_TRACE
+          if (blockIdx.x == 0 && n == 1 && j < 64 && lane == 0) g_trace_w[((warp - kFirstSoftmaxWarp) * 64 + j) * 2] = clock64();
+#endif
           if (nk == 128) softmax_slab<128>(tS, tO, m, first, g.scale_log2, m_ref, l, bh, br, tr);
           else if (nk == 112) softmax_slab<112>(tS, tO, m, first, g.scale_log2, m_ref, l, bh, br, tr);
           else if (nk == 96) softmax_slab<96>(tS, tO, m, first, g.scale_log2, m_ref, l, bh, br, tr);
           else softmax_slab<64>(tS, tO, m, first, g.scale_log2, m_ref, l, bh, br, tr);
           TRACE(qi, j, 4);
+#ifdef PSA_TRACE
+          if (blockIdx.x == 0 && n == 1 && j < 64 && lane == 0) g_trace_w[((warp - kFirstSoftmaxWarp) * 64 + j) * 2 + 1] = clock64();
+#endif
         }
       }
       kv_g += (uint32_t)n_kv;
@@ -1106,7 +1164,7 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
   if (threadIdx.x == 0 && *abort_flag != 0) {
     if (atomicCAS(prm.ws_header + kWsStatus, 0, (int)PSA_ERR_TIMEOUT) == 0) prm.ws_header[kWsDetail] = *abort_flag;
   }
-  if (warp == 9) {
+  if (warp == kWarpMma) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(*tmem_slot), "r"(512) : "memory");
   }
@@ -1175,6 +1233,9 @@ cudaError_t launch_attn(const TensorMaps& tm, const Geom& g, const WorkItem* ite
 #ifdef PSA_TRACE
 extern "C" int psa_debug_read_trace(long long* out, int n) {
   return (int)cudaMemcpyFromSymbol(out, psa::g_trace, sizeof(long long) * n);
+}
+extern "C" int psa_debug_read_trace_w(long long* out, int n) {
+  return (int)cudaMemcpyFromSymbol(out, psa::g_trace_w, sizeof(long long) * n);
 }
 extern "C" int psa_debug_read_items(long long* out, int n) {
   return (int)cudaMemcpyFromSymbol(out, psa::g_trace_items, sizeof(long long) * n);
