@@ -9,19 +9,21 @@
 // the even and the odd key slabs, and their partial results are merged in the epilogue.
 //
 // Roles (384 threads = 3 warpgroups):
-//   warps 0-3  softmax / correction / epilogue of tile 0 = (S0, O0)   (TMEM lanes 0..127)
-//   warps 4-7  the same for tile 1 = (S1, O1)
-//   warp  8    scheduler + TMA loads: Q slabs once per item, K and V slabs through a 5-slot ring
+//   warp  0    tcgen05.mma issue: S_i = Q_i K^T (SS form), O_i += P_i V (P read from TMEM).  Its
+//              own instruction stream is on the critical path, so it probes two barriers per
+//              shared-memory round trip and divides nothing inside the loop
+//   warp  1    scheduler + TMA loads: Q slabs once per item, K and V slabs through a 5-slot ring
 //              (V_j travels with K_{j+1} under one barrier)
-//   warp  9    tcgen05.mma issue: S_i = Q_i K^T (SS form), O_i += P_i V (P read from TMEM)
-//   warps 10-11 idle; they only exist so that the third warpgroup can hand its registers
+//   warps 2-3  idle; they only exist so that the first warpgroup can hand its registers
 //              to the softmax warpgroups (setmaxnreg)
+//   warps 4-7  softmax / correction / epilogue of tile 0 = (S0, O0)   (TMEM lanes 0..127)
+//   warps 8-11 the same for tile 1 = (S1, O1)
 // TMEM (512 columns): S0 | S1 | O0 | O1, 128 fp32 columns each; the bf16 probabilities
 // P_i overwrite the first columns of S_i.  A key slab has 128 keys, or 112/96/64 for the last
 // slab of a block whose token count is not a multiple of 128.
 // Every wait is bounded; on expiry the CTA records a status word and unwinds.
-// Build-time knobs: PSA_EMU_PAIRS (share of
-// exponentials computed by a polynomial on the FMA pipe, default 0), PSA_TRACE (cycle stamps).
+// Build-time knobs: PSA_EMU_PAIRS (share of exponentials computed by a polynomial on the FMA
+// pipe, default 0), PSA_TRACE (cycle stamps).
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -30,11 +32,7 @@
 namespace psa {
 
 constexpr int kThreads = 384;                       // 3 warpgroups; register budgets are re-split below
-#if !defined(PSA_UTIL_FIRST) || PSA_UTIL_FIRST
-constexpr int kWarpMma = 0, kWarpLoad = 1, kUtilGroup = 0, kFirstSoftmaxWarp = 4;
-#else
-constexpr int kWarpMma = 9, kWarpLoad = 8, kUtilGroup = 2, kFirstSoftmaxWarp = 0;
-#endif
+constexpr int kWarpMma = 0, kWarpLoad = 1, kUtilGroup = 0, kFirstSoftmaxWarp = 4;   // warp roles
 constexpr int kNumSlots = 5;                       // K/V ring slots of one 128 x 128 bf16 slab
 constexpr uint32_t kSlabBytes = 128 * 128 * 2;     // 32 KB
 constexpr uint32_t kHalfBytes = kSlabBytes / 2;    // one 64-column swizzled half
@@ -283,9 +281,6 @@ __device__ __forceinline__ void exp2_poly_pair(uint64_t x2, float& p0, float& p1
 }
 #ifndef PSA_EMU_PAIRS
 #define PSA_EMU_PAIRS 0   // of every 4 pairs of probabilities, this many use exp2_poly_pair (0: all ex2.approx)
-#endif
-#ifndef PSA_UTIL_FIRST
-#define PSA_UTIL_FIRST 1  // 1: MMA and load warps are warps 0 and 1 (oldest warps of their schedulers); 0: warps 9 and 8
 #endif
 
 
@@ -602,7 +597,7 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
   };
 
   if ((warp >> 2) == kUtilGroup) {
-  // Third warpgroup: give registers away (the budget is re-split per warpgroup).
+  // Utility warpgroup: give registers away (the budget is re-split per warpgroup).
   asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
   if (warp == kWarpLoad) {
     // ======================================================================= load warp
@@ -876,18 +871,17 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
         int rj = 0;   // residue of slab j; r0 is that of slab j + 2 from here on
         for (int j = 0; ok && j < n_kv; ++j) {
           const int i = j & 1;
-          ok = mbar_wait_warp(bar(kBarPairFull + pair_g % kNumPairBars), (pair_g / kNumPairBars) & 1u, abort_flag, 0x231);
+          const uint32_t cs = i == 0 ? cnt_s0 : cnt_s1;
+          ok = mbar_wait2_warp(bar(kBarPairFull + pair_g % kNumPairBars), (pair_g / kNumPairBars) & 1u,
+                               bar(kBarPHalf + i), cs & 1u, abort_flag, 0x231, 0x234 + i);
           if (!ok) break;
           ++pair_g;
           const bool more = (j + 2 < n_kv);
           const uint32_t vslot = tile_g % kNumSlots;
           const uint32_t kslot = (tile_g + 1) % kNumSlots;
           tile_g += more ? 2u : 1u;
-          const uint32_t cs = i == 0 ? cnt_s0 : cnt_s1;
           const int nk_cur = nk_at(rj);
           rj = r_inc(rj);
-          ok = mbar_wait_warp(bar(kBarPHalf + i), cs & 1u, abort_flag, 0x234 + i);
-          if (!ok) break;
           tc_fence_after();
           if (elect_one()) issue_pv_half(i, vslot, 0, j > 1, nk_cur);
           ok = mbar_wait_warp(bar(kBarPReady + i), cs & 1u, abort_flag, 0x232 + i);
