@@ -137,6 +137,16 @@ int psa_attn_fwd_host(const void* q, const void* k, const void* v, void* out, fl
                       const psa_head_params* head_params, const psa_problem* prob,
                       int T, int H, int W, void* stream);
 
+/* Batched call (what one DiT attention layer issues: batch > 1, or the conditional / unconditional
+ * pair of classifier-free guidance).  The paper assigns masks per head, not per sample, so all
+ * n_batch samples use the same head_params.  Element (b, head, token, c) of q, k, v, out sits at
+ * b*stride_batch + head*stride_head + token*stride_token + c; lse is [n_batch][n_heads][L].
+ * When the batches are evenly spaced heads (stride_batch == n_heads*stride_head) all samples run in
+ * one launch sequence, otherwise sample by sample.  Everything else as psa_attn_fwd. */
+int psa_attn_fwd_batched(const void* q, const void* k, const void* v, void* out, float* lse,
+                         const psa_head_params* head_params, const psa_problem* prob, int n_batch,
+                         int64_t stride_batch, int T, int H, int W, void* stream);
+
 /* PSA-Search for ONE head (Appendix C, Algorithm 3).
  *
  * psa_search_losses: the inner loop -- Loss(M) = L2Loss(PSA(h, M), FullAttn(h)) for every candidate

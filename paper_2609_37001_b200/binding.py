@@ -64,6 +64,7 @@ def lib() -> ctypes.CDLL:
         L.psa_attn_fwd_host.argtypes = [vp] * 10 + [hp, pp, i32, i32, i32, vp]
         L.psa_attn_fwd_noalloc.argtypes = [vp, vp, vp, vp, vp, hp, pp, i32, i32, i32, vp, ctypes.POINTER(ctypes.c_int32)]
         L.psa_attn_fwd_noalloc.restype = ctypes.c_int
+        L.psa_attn_fwd_batched.argtypes = [vp, vp, vp, vp, vp, hp, pp, i32, ctypes.c_int64, i32, i32, i32, vp]
         L.psa_search_scratch_bytes.argtypes = [i32, i32, i32, i32]
         L.psa_search_scratch_bytes.restype = ctypes.c_int64
         L.psa_search_losses.argtypes = [vp, vp, vp, hp, i32, pp, i32, i32, i32, vp, vp, vp]
@@ -186,6 +187,34 @@ def psa_attn_fwd(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, head_params,
     _check(lib().psa_attn_fwd(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), lse.data_ptr(),
                               _params_array(head_params), ctypes.byref(prob), T, H, W, _stream_ptr(stream)),
            "psa_attn_fwd")
+    return out, lse
+
+
+def psa_attn_fwd_batched(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, head_params, grid: Sequence[int],
+                         tile: Sequence[int], scale: float, out: Optional[torch.Tensor] = None,
+                         lse: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None):
+    """Batched call: q, k, v are bf16 device tensors [batch, heads, L, 128] sharing strides (last dim
+    contiguous); every sample uses the same per-head masks.  Returns (out like q, lse fp32
+    [batch, heads, L])."""
+    _require_cuda(q, k, v)
+    if q.dtype != torch.bfloat16 or k.dtype != torch.bfloat16 or v.dtype != torch.bfloat16:
+        raise ValueError("bf16 tensors required")
+    nb, nh, L, d = q.shape
+    T, H, W = (int(x) for x in grid)
+    if L != T * H * W or k.shape != q.shape or v.shape != q.shape or len(head_params) != nh:
+        raise ValueError("shape mismatch")
+    if q.stride() != k.stride() or q.stride() != v.stride() or q.stride(3) != 1:
+        raise ValueError("q, k, v must share strides with a contiguous last dimension")
+    if out is None:
+        out = torch.empty_strided(q.shape, q.stride(), dtype=q.dtype, device=q.device)
+    if lse is None:
+        lse = torch.empty((nb, nh, L), dtype=torch.float32, device=q.device)
+    if out.stride() != q.stride() or not lse.is_contiguous():
+        raise ValueError("out must share q's strides; lse must be contiguous")
+    prob = make_problem(nh, tile, scale, q.stride(1), q.stride(2), d)
+    _check(lib().psa_attn_fwd_batched(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), lse.data_ptr(),
+                                      _params_array(head_params), ctypes.byref(prob), nb, q.stride(0), T, H, W,
+                                      _stream_ptr(stream)), "psa_attn_fwd_batched")
     return out, lse
 
 

@@ -410,6 +410,46 @@ int psa_search_select_at_sparsity(const float* losses, const float* sparsity, in
   return best < 0 ? PSA_ERR_CAPACITY : best;
 }
 
+int psa_attn_fwd_batched(const void* q, const void* k, const void* v, void* out, float* lse,
+                         const psa_head_params* head_params, const psa_problem* prob, int n_batch, int64_t stride_batch,
+                         int T, int H, int W, void* stream) {
+  Geom g;
+  int rc = make_geom(prob, T, H, W, true, &g);
+  if (rc != PSA_OK) return rc;
+  if (!q || !k || !v || !out || !lse || !head_params || n_batch < 1) return PSA_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || (reinterpret_cast<uintptr_t>(lse) & 3u))
+    return PSA_ERR_INVALID_ARG;
+  if (out == q || out == k || out == v) return PSA_ERR_INVALID_ARG;
+  if (prob->stride_token < kHeadDim || (prob->stride_token % 8) != 0) return PSA_ERR_INVALID_ARG;
+  if (prob->n_heads > 1 && (prob->stride_head < kHeadDim || (prob->stride_head % 8) != 0)) return PSA_ERR_INVALID_ARG;
+  if (n_batch > 1 && (stride_batch < kHeadDim || (stride_batch % 8) != 0)) return PSA_ERR_INVALID_ARG;
+  for (int h = 0; h < prob->n_heads; ++h)
+    if (!valid_params(head_params[h])) return PSA_ERR_INVALID_ARG;
+  const int nh = prob->n_heads;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  std::lock_guard<std::mutex> lock(g_mu);
+  const bool fold = n_batch == 1 || (nh == 1 ? true : stride_batch == (int64_t)nh * prob->stride_head);
+  if (fold) {
+    // samples are evenly spaced heads: one launch sequence over n_batch * n_heads heads
+    if ((long long)n_batch * nh >= (1ll << 24)) return PSA_ERR_UNSUPPORTED;
+    std::vector<psa_head_params> params((size_t)n_batch * nh);
+    for (int b = 0; b < n_batch; ++b)
+      for (int h = 0; h < nh; ++h) params[(size_t)b * nh + h] = head_params[h];
+    const long long hs = nh == 1 ? (n_batch > 1 ? stride_batch : prob->stride_head) : prob->stride_head;
+    const Layout lay = {hs, prob->stride_token, hs, prob->stride_token, false};
+    return run_attn(q, k, v, out, lse, params.data(), n_batch * nh, g, lay, st);
+  }
+  const Layout lay = {prob->stride_head, prob->stride_token, prob->stride_head, prob->stride_token, false};
+  for (int b = 0; b < n_batch; ++b) {
+    const long long off = (long long)b * stride_batch;
+    rc = run_attn(static_cast<const uint16_t*>(q) + off, static_cast<const uint16_t*>(k) + off,
+                  static_cast<const uint16_t*>(v) + off, static_cast<uint16_t*>(out) + off,
+                  lse + (long long)b * nh * g.L, head_params, nh, g, lay, st);
+    if (rc != PSA_OK) return rc;
+  }
+  return PSA_OK;
+}
+
 // ---- PSA-Search for one head (Algorithm 3) ------------------------------------------------------
 // scratch layout: outputs of the n_cand candidates and of full attention ((n_cand + 1) x L x 128 bf16),
 // their lse ((n_cand + 1) x L fp32), the partial sums of the loss reduction.

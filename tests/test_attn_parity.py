@@ -203,3 +203,35 @@ def test_more_heads_than_one_launch_carries(B):
         qf, kf, vf = (O.bf16_bits_to_f64(bits[n][hd]) for n in ("q", "k", "v"))
         ro, rl = O.attention(qf, kf, vf, params[hd], *grid, tile, SCALE)
         _compare(_bf16_to_f64(out[hd]), lse[hd].cpu().numpy().astype(np.float64), ro, rl, f"head {hd}")
+
+
+@pytest.mark.parametrize("even_spacing", [True, False])
+def test_batched_call_matches_oracle_per_sample(B, even_spacing):
+    """psa_attn_fwd_batched: a conditional / unconditional pair with shared per-head masks, once with the
+    samples laid out as evenly spaced heads (one launch sequence) and once with a padded batch stride
+    (sample by sample)."""
+    grid, tile = (4, 12, 16), (1, 8, 16)
+    T, H, W = grid
+    L, nb, nh = T * H * W, 2, 3
+    params = [(2, 0, INF, 2, 0, INF), (1, 1, 2, 3, 0, INF), (4, 0, INF, 1, 0, 2)]
+    bits = {n: WL.tensor_bits(77, n, nb * nh, L) for n in ("q", "k", "v")}
+
+    def dev(n):
+        full = _to_dev(bits[n]).view(nb, nh, L, 128)
+        if even_spacing:
+            return full
+        buf = torch.zeros((nb, nh + 1, L, 128), dtype=torch.bfloat16, device="cuda")
+        buf[:, :nh] = full
+        return buf[:, :nh]
+
+    q, k, v = dev("q"), dev("k"), dev("v")
+    out, lse = B.psa_attn_fwd_batched(q, k, v, params, grid, tile, SCALE)
+    st, detail = B.psa_last_device_status()
+    assert st == 0, (st, hex(detail))
+    out_h = _bf16_to_f64(out).reshape(nb, nh, L, 128)
+    lse_h = lse.cpu().numpy().astype(np.float64)
+    for b in range(nb):
+        for hd in range(nh):
+            qf, kf, vf = (O.bf16_bits_to_f64(bits[n][b * nh + hd]) for n in ("q", "k", "v"))
+            ro, rl = O.attention(qf, kf, vf, params[hd], T, H, W, tuple(tile), SCALE)
+            _compare(out_h[b, hd], lse_h[b, hd], ro, rl, f"sample {b} head {hd}")
