@@ -281,6 +281,45 @@ def attention(q: np.ndarray, k: np.ndarray, v: np.ndarray, params: Params,
     return attention_rows(q, k, v, range(q.shape[0]), params, T, H, W, tile, scale)
 
 
+def attend_row_with_text(i: int, params: Params, tb: np.ndarray, sb: np.ndarray, n_text: int) -> np.ndarray:
+    """Attended keys of query i when n_text text tokens follow the L video tokens (a multimodal DiT's
+    joint sequence).  The paper defines the stripe mask on the video grid only and does not say how the
+    text tokens are treated; the reading taken: the mask applies between video tokens, every query
+    attends every text key, and a text query attends every key."""
+    L = tb.shape[0]
+    att = np.ones(L + n_text, dtype=bool)
+    if i < L:
+        att[:L] = attend_row(i, params, tb, sb)
+    return att
+
+
+def attention_rows_with_text(q: np.ndarray, k: np.ndarray, v: np.ndarray, rows: Iterable[int], params: Params,
+                             T: int, H: int, W: int, tile: Tile, scale: float, n_text: int):
+    """Masked attention over the joint sequence: q, k, v are float64 [L + n_text, d], video tokens first.
+    Returns (out float64[len(rows), d], lse float64[len(rows)]) for the query tokens in ``rows``."""
+    rows = np.asarray(list(rows), dtype=np.int64)
+    tb, sb, _ = token_block_coords(T, H, W, tile)
+    out = np.zeros((rows.size, q.shape[1]), dtype=np.float64)
+    lse = np.full(rows.size, -np.inf, dtype=np.float64)
+    for r, i in enumerate(rows):
+        idx = np.flatnonzero(attend_row_with_text(int(i), params, tb, sb, n_text))
+        if idx.size == 0:
+            continue
+        a = scale * (k[idx] @ q[i])
+        m = a.max()
+        e = np.exp(a - m)
+        l = e.sum()
+        out[r] = (e @ v[idx]) / l
+        lse[r] = m + math.log(l)
+    return out, lse
+
+
+def attention_with_text(q: np.ndarray, k: np.ndarray, v: np.ndarray, params: Params,
+                        T: int, H: int, W: int, tile: Tile, scale: float, n_text: int):
+    """All rows of attention_rows_with_text."""
+    return attention_rows_with_text(q, k, v, range(q.shape[0]), params, T, H, W, tile, scale, n_text)
+
+
 def dense_attention(q: np.ndarray, k: np.ndarray, v: np.ndarray, scale: float):
     """Unmasked softmax attention of one head, written without any mask logic."""
     a = scale * (q @ k.T)
