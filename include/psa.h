@@ -147,6 +147,22 @@ int psa_attn_fwd_batched(const void* q, const void* k, const void* v, void* out,
                          const psa_head_params* head_params, const psa_problem* prob, int n_batch,
                          int64_t stride_batch, int T, int H, int W, void* stream);
 
+/* Joint video + text sequence (multimodal DiT blocks such as HunyuanVideo's, which attend over the
+ * video tokens and the prompt's text tokens together).  The paper defines the stripe mask on the video
+ * grid and is silent on the text tokens; the reading taken: the mask applies between video tokens,
+ * every query attends every text key, and a text query attends every key.
+ *   q, k, v, out  device bf16; every head holds L = T*H*W video tokens followed by n_text text tokens
+ *                 (token index L .. L+n_text-1), element (head, token, c) at
+ *                 head*stride_head + token*stride_token + c
+ *   lse           device fp32 [n_heads][L + n_text]
+ *   n_text        >= 0 (0 is psa_attn_fwd); at most 65535 * 128
+ * Text keys travel as extra 128-token key slabs after the attended video slabs of every work item
+ * (a ragged last slab is zero-filled and masked); text queries are extra work items that attend all
+ * key blocks.  Everything else as psa_attn_fwd. */
+int psa_attn_fwd_joint(const void* q, const void* k, const void* v, void* out, float* lse,
+                       const psa_head_params* head_params, const psa_problem* prob, int64_t n_text,
+                       int T, int H, int W, void* stream);
+
 /* PSA-Search for ONE head (Appendix C, Algorithm 3).
  *
  * psa_search_losses: the inner loop -- Loss(M) = L2Loss(PSA(h, M), FullAttn(h)) for every candidate

@@ -65,6 +65,7 @@ def lib() -> ctypes.CDLL:
         L.psa_attn_fwd_noalloc.argtypes = [vp, vp, vp, vp, vp, hp, pp, i32, i32, i32, vp, ctypes.POINTER(ctypes.c_int32)]
         L.psa_attn_fwd_noalloc.restype = ctypes.c_int
         L.psa_attn_fwd_batched.argtypes = [vp, vp, vp, vp, vp, hp, pp, i32, ctypes.c_int64, i32, i32, i32, vp]
+        L.psa_attn_fwd_joint.argtypes = [vp, vp, vp, vp, vp, hp, pp, ctypes.c_int64, i32, i32, i32, vp]
         L.psa_search_scratch_bytes.argtypes = [i32, i32, i32, i32]
         L.psa_search_scratch_bytes.restype = ctypes.c_int64
         L.psa_search_losses.argtypes = [vp, vp, vp, hp, i32, pp, i32, i32, i32, vp, vp, vp]
@@ -215,6 +216,34 @@ def psa_attn_fwd_batched(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, head
     _check(lib().psa_attn_fwd_batched(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), lse.data_ptr(),
                                       _params_array(head_params), ctypes.byref(prob), nb, q.stride(0), T, H, W,
                                       _stream_ptr(stream)), "psa_attn_fwd_batched")
+    return out, lse
+
+
+def psa_attn_fwd_joint(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, head_params, grid: Sequence[int],
+                       tile: Sequence[int], scale: float, n_text: int, out: Optional[torch.Tensor] = None,
+                       lse: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None):
+    """Joint video + text sequence: q, k, v are bf16 device tensors [heads, L + n_text, 128] with the
+    video tokens first.  The stripe mask applies between video tokens; text keys are attended by every
+    query and text queries attend every key.  Returns (out like q, lse fp32 [heads, L + n_text])."""
+    _require_cuda(q, k, v)
+    if q.dtype != torch.bfloat16 or k.dtype != torch.bfloat16 or v.dtype != torch.bfloat16:
+        raise ValueError("bf16 tensors required")
+    nh, Lt, d = q.shape
+    T, H, W = (int(x) for x in grid)
+    if Lt != T * H * W + int(n_text) or k.shape != q.shape or v.shape != q.shape:
+        raise ValueError("shape mismatch")
+    if q.stride() != k.stride() or q.stride() != v.stride() or q.stride(2) != 1:
+        raise ValueError("q, k, v must share strides with a contiguous last dimension")
+    if out is None:
+        out = torch.empty_strided(q.shape, q.stride(), dtype=q.dtype, device=q.device)
+    if lse is None:
+        lse = torch.empty((nh, Lt), dtype=torch.float32, device=q.device)
+    if out.stride() != q.stride() or not lse.is_contiguous():
+        raise ValueError("out must share q's strides; lse must be contiguous")
+    prob = make_problem(nh, tile, scale, q.stride(0), q.stride(1), d)
+    _check(lib().psa_attn_fwd_joint(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), lse.data_ptr(),
+                                    _params_array(head_params), ctypes.byref(prob), int(n_text), T, H, W,
+                                    _stream_ptr(stream)), "psa_attn_fwd_joint")
     return out, lse
 
 

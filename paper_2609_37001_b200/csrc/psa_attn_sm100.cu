@@ -345,7 +345,15 @@ plan_kernel(const HeadParamsArray hp, const Geom g, int head0, int* __restrict__
   for (int qb = threadIdx.x; qb < g.NB; qb += blockDim.x) cnt[qb] = cntT[qb / g.Sp] * cntS[qb % g.Sp];
   __syncthreads();
   const int ipb = g.items_per_block;
-  WorkItem* out = items + (size_t)h * g.NB * ipb;
+  // Text-query items first: they attend every key block, so they are the heaviest of the head.
+  // Two text slabs per item; a single one runs in split-KV mode.  Flag in bit 25.
+  WorkItem* head_items = items + (size_t)h * g.items_per_head;
+  for (int it = threadIdx.x; it < g.n_titems; it += blockDim.x) {
+    const int sub0 = 2 * it;
+    const int nq = (g.n_ts - sub0) >= 2 ? 2 : 1;
+    head_items[it] = make_int4(h, 0, g.NB, sub0 | (nq << 16) | ((nq == 1 ? 1 : 0) << 24) | (1 << 25));
+  }
+  WorkItem* out = head_items + g.n_titems;
   for (int qb = threadIdx.x; qb < g.NB; qb += blockDim.x) {
     const int c = cnt[qb];
     int rank = 0;
@@ -377,7 +385,7 @@ struct AttnParams {
 };
 
 struct TensorMaps {
-  CUtensorMap q[2], k[2], v[2], o[2];  // [0]: full 128-token slab box, [1]: a block's last slab
+  CUtensorMap q[3], k[3], v[3], o[3];  // [0]: full 128-token slab box, [1]: a block's last slab, [2]: text slab
 };
 
 // Extents and token count of slab `sub` of a block; `last` selects the tensor-map set.
@@ -625,19 +633,20 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
       wi.w = __shfl_sync(0xffffffffu, wi.w, 0);
       if (wi.x < 0) break;
       const int head = wi.x, qb = wi.y, sub0 = wi.w & 0xffff, nq = (wi.w >> 16) & 0xff;
-      const int lag = (wi.w >> 24) ? 2 : 1;   // V_j travels with K_{j+lag} (2 in split-KV mode)
+      const int lag = ((wi.w >> 24) & 1) ? 2 : 1;   // V_j travels with K_{j+lag} (2 in split-KV mode)
+      const bool textq = ((wi.w >> 25) & 1) != 0;   // the queries are text tokens: every key is attended
       const int head_ld = prm.shared_qkv ? 0 : head;   // head coordinate of the q, k, v loads
       const psa_head_params p = prm.hp_dev[head];
       const int tq = qb / g.Sp, sq = qb % g.Sp;
       // attended key-block coordinates of this query block, one bit per block coordinate
       for (int b = 0; b < g.Tp; b += 32) {
         const int tk = b + lane;
-        const unsigned m = __ballot_sync(0xffffffffu, tk < g.Tp && axis_attends(tk - tq, p.Tw, p.To, p.Ts));
+        const unsigned m = __ballot_sync(0xffffffffu, tk < g.Tp && (textq || axis_attends(tk - tq, p.Tw, p.To, p.Ts)));
         if (lane == 0) maskT[b >> 5] = m;
       }
       for (int b = 0; b < g.Sp; b += 32) {
         const int sk = b + lane;
-        const unsigned m = __ballot_sync(0xffffffffu, sk < g.Sp && axis_attends(sk - sq, p.Sw, p.So, p.Ss));
+        const unsigned m = __ballot_sync(0xffffffffu, sk < g.Sp && (textq || axis_attends(sk - sq, p.Sw, p.So, p.Ss)));
         if (lane == 0) maskS[b >> 5] = m;
       }
       __syncwarp();
@@ -650,8 +659,12 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
         if (!ok) break;
         if (lane == 0) {
           int t0, h0, w0, et, eh, ew, ntok, last;
-          slab_origin(g, qb, sub0 + i, t0, h0, w0);
-          slab_shape(g, sub0 + i, et, eh, ew, ntok, last);
+          if (textq) {   // text slab: 128 tokens from the text map, token index in the second coordinate
+            t0 = 0; h0 = 0; w0 = (sub0 + i) * kSlabTokens; ntok = kSlabTokens; last = 2;
+          } else {
+            slab_origin(g, qb, sub0 + i, t0, h0, w0);
+            slab_shape(g, sub0 + i, et, eh, ew, ntok, last);
+          }
           const uint32_t dst = sbase + kOffQ + (uint32_t)i * kSlabBytes;
           mbar_expect_tx(bar(kBarQFull + i), (uint32_t)ntok * 256u);
           tma_load_5d(dst, &tms.q[last], bar(kBarQFull + i), 0, w0, h0, t0, head_ld);
@@ -664,6 +677,46 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
       int npend = 0;
       int at0 = 0, ah0 = 0, aw0 = 0, alast = 0, antok = kSlabTokens;  // oldest pending slab
       int bt0 = 0, bh0 = 0, bw0 = 0, blast = 0, bntok = kSlabTokens;  // newer pending slab (lag 2)
+      // One key slab: K now, V of the slab issued `lag` slabs earlier under the same barrier.
+      auto issue_slab = [&](int t0, int h0, int w0, int last, int ntok, uint32_t vw0, uint32_t vw1, uint32_t vw2,
+                            uint32_t vw3) {
+        // slots: [V of the oldest pending slab,] K of this slab
+        const bool with_v = (npend == lag);
+        const uint32_t v_slot = tile_g % kNumSlots, v_use = tile_g / kNumSlots;
+        const uint32_t k_tile = tile_g + (with_v ? 1u : 0u);
+        const uint32_t k_slot = k_tile % kNumSlots, k_use = k_tile / kNumSlots;
+        if (with_v) {
+          ok = mbar_wait_warp(bar(kBarSlotEmpty + v_slot), (v_use & 1u) ^ 1u, abort_flag, 0x111);
+          if (!ok) return;
+        }
+        ok = mbar_wait_warp(bar(kBarSlotEmpty + k_slot), (k_use & 1u) ^ 1u, abort_flag, 0x110);
+        if (!ok) return;
+        if (lane == 0) {
+          uint32_t* m = meta + (kv_g % kMetaRing) * 8;
+          m[0] = vw0; m[1] = vw1; m[2] = vw2; m[3] = vw3;
+          const uint32_t pb = bar(kBarPairFull + pair_g % kNumPairBars);
+          mbar_expect_tx(pb, (uint32_t)((with_v ? antok : 0) + ntok) * 256u);
+          if (with_v) {
+            const uint32_t dv = sbase + kOffRing + v_slot * kSlabBytes;
+            tma_load_5d(dv, &tms.v[alast], pb, 0, aw0, ah0, at0, head_ld);
+            tma_load_5d(dv + kHalfBytes, &tms.v[alast], pb, 64, aw0, ah0, at0, head_ld);
+          }
+          const uint32_t dk = sbase + kOffRing + k_slot * kSlabBytes;
+          tma_load_5d(dk, &tms.k[last], pb, 0, w0, h0, t0, head_ld);
+          tma_load_5d(dk + kHalfBytes, &tms.k[last], pb, 64, w0, h0, t0, head_ld);
+        }
+        tile_g = k_tile + 1;
+        ++pair_g;
+        ++kv_g;
+        // queue this slab's V
+        if (with_v) {
+          if (lag == 2) { at0 = bt0; ah0 = bh0; aw0 = bw0; alast = blast; antok = bntok; }
+          --npend;
+        }
+        if (npend == 0) { at0 = t0; ah0 = h0; aw0 = w0; alast = last; antok = ntok; }
+        else { bt0 = t0; bh0 = h0; bw0 = w0; blast = last; bntok = ntok; }
+        ++npend;
+      };
       for (int tw = 0; ok && tw < g.Tp; tw += 32) {
         uint32_t mt = maskT[tw >> 5];
         while (ok && mt) {
@@ -693,46 +746,21 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
                   c += 32;
                   vw3 = __ballot_sync(0xffffffffu, (t0 + c / ehw < g.T) && (h0 + (c / ew) % eh < g.H) && (w0 + c % ew < g.W));
                 }
-                // slots: [V of the oldest pending slab,] K of this slab
-                const bool with_v = (npend == lag);
-                const uint32_t v_slot = tile_g % kNumSlots, v_use = tile_g / kNumSlots;
-                const uint32_t k_tile = tile_g + (with_v ? 1u : 0u);
-                const uint32_t k_slot = k_tile % kNumSlots, k_use = k_tile / kNumSlots;
-                if (with_v) {
-                  ok = mbar_wait_warp(bar(kBarSlotEmpty + v_slot), (v_use & 1u) ^ 1u, abort_flag, 0x111);
-                  if (!ok) break;
-                }
-                ok = mbar_wait_warp(bar(kBarSlotEmpty + k_slot), (k_use & 1u) ^ 1u, abort_flag, 0x110);
-                if (!ok) break;
-                if (lane == 0) {
-                  uint32_t* m = meta + (kv_g % kMetaRing) * 8;
-                  m[0] = vw0; m[1] = vw1; m[2] = vw2; m[3] = vw3;
-                  const uint32_t pb = bar(kBarPairFull + pair_g % kNumPairBars);
-                  mbar_expect_tx(pb, (uint32_t)((with_v ? antok : 0) + ntok) * 256u);
-                  if (with_v) {
-                    const uint32_t dv = sbase + kOffRing + v_slot * kSlabBytes;
-                    tma_load_5d(dv, &tms.v[alast], pb, 0, aw0, ah0, at0, head_ld);
-                    tma_load_5d(dv + kHalfBytes, &tms.v[alast], pb, 64, aw0, ah0, at0, head_ld);
-                  }
-                  const uint32_t dk = sbase + kOffRing + k_slot * kSlabBytes;
-                  tma_load_5d(dk, &tms.k[last], pb, 0, w0, h0, t0, head_ld);
-                  tma_load_5d(dk + kHalfBytes, &tms.k[last], pb, 64, w0, h0, t0, head_ld);
-                }
-                tile_g = k_tile + 1;
-                ++pair_g;
-                ++kv_g;
-                // queue this slab's V
-                if (with_v) {
-                  if (lag == 2) { at0 = bt0; ah0 = bh0; aw0 = bw0; alast = blast; antok = bntok; }
-                  --npend;
-                }
-                if (npend == 0) { at0 = t0; ah0 = h0; aw0 = w0; alast = last; antok = ntok; }
-                else { bt0 = t0; bh0 = h0; bw0 = w0; blast = last; bntok = ntok; }
-                ++npend;
+                issue_slab(t0, h0, w0, last, ntok, vw0, vw1, vw2, vw3);
               }
             }
           }
         }
+      }
+      // text key slabs: attended by every query; tokens beyond n_text are zero-filled and masked
+      for (int ts = 0; ok && ts < g.n_ts; ++ts) {
+        const int tok0 = ts * kSlabTokens;
+        const int nvalid = g.n_text - tok0;   // >= 1
+        const uint32_t vw0 = nvalid >= 32 ? 0xffffffffu : ((1u << nvalid) - 1u);
+        const uint32_t vw1 = nvalid >= 64 ? 0xffffffffu : (nvalid <= 32 ? 0u : ((1u << (nvalid - 32)) - 1u));
+        const uint32_t vw2 = nvalid >= 96 ? 0xffffffffu : (nvalid <= 64 ? 0u : ((1u << (nvalid - 64)) - 1u));
+        const uint32_t vw3 = nvalid >= 128 ? 0xffffffffu : (nvalid <= 96 ? 0u : ((1u << (nvalid - 96)) - 1u));
+        issue_slab(0, 0, tok0, 2, kSlabTokens, vw0, vw1, vw2, vw3);
       }
       while (ok && npend > 0) {  // V of the item's last slab(s), one pair barrier each
         const uint32_t v_slot = tile_g % kNumSlots, v_use = tile_g / kNumSlots;
@@ -823,8 +851,10 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
       WorkItem wi;
       if (!next_item(n, wi)) break;
       const int nq = (wi.w >> 16) & 0xff;
-      const bool split = (wi.w >> 24) != 0;
-      const int n_kv = wi.z * g.n_sub;
+      const bool split = ((wi.w >> 24) & 1) != 0;
+      const int n_vid = wi.z * g.n_sub;          // video key slabs, then the text slabs (always 128 wide)
+      const int n_kv = n_vid + g.n_ts;
+      auto nk_j = [&](int j, int r) -> int { return j >= n_vid ? kSlabTokens : nk_at(r); };
 #ifdef PSA_TRACE
       if ((blockIdx.x == 0 || blockIdx.x == 77) && n < 256 && lane == 0) {
         long long* r = g_trace_items + ((blockIdx.x == 0 ? 0 : 1) * 256 + n) * 4;
@@ -861,7 +891,7 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
           ++tile_g;
           tc_fence_after();
           if (elect_one()) {
-            issue_qk(0, slot, nk_at(r0), j);
+            issue_qk(0, slot, nk_j(j, r0), j);
             tc_commit(bar(kBarSFull + j));
             tc_commit(bar(kBarSlotEmpty + slot));
           }
@@ -880,7 +910,7 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
           const uint32_t vslot = tile_g % kNumSlots;
           const uint32_t kslot = (tile_g + 1) % kNumSlots;
           tile_g += more ? 2u : 1u;
-          const int nk_cur = nk_at(rj);
+          const int nk_cur = nk_j(j, rj);
           rj = r_inc(rj);
           tc_fence_after();
           if (elect_one()) issue_pv_half(i, vslot, 0, j > 1, nk_cur);
@@ -892,7 +922,7 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
             issue_pv_half(i, vslot, 1, true, nk_cur);
             tc_commit(bar(kBarSlotEmpty + vslot));
             if (more) {
-              issue_qk(0, kslot, nk_at(r0), i);
+              issue_qk(0, kslot, nk_j(j + 2, r0), i);
               r0 = r_inc(r0);
               tc_commit(bar(kBarSFull + i));
               tc_commit(bar(kBarSlotEmpty + kslot));
@@ -916,7 +946,7 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
 #pragma unroll
             for (int i = 0; i < 2; ++i) {
               if (i < nq) {
-                issue_qk(i, slot, nk_at(0), i);
+                issue_qk(i, slot, nk_j(0, 0), i);
                 tc_commit(bar(kBarSFull + i));
               }
             }
@@ -926,9 +956,9 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
         }
         int rj = 0;
         for (int j = 0; ok && j < n_kv; ++j) {
-          const int nk_cur = nk_at(rj);
+          const int nk_cur = nk_j(j, rj);
           rj = r_inc(rj);
-          const int nk_next = nk_at(rj);
+          const int nk_next = nk_j(j + 1, rj);
           // V_j and (unless this is the last slab) K_{j+1} arrive under one barrier; it is waited
           // for together with the first half of P_0 (one shared-memory round trip for both)
           TRACE(2, j, 5);
@@ -1009,8 +1039,10 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
       WorkItem wi;
       if (!next_item(n, wi)) break;
       const int head = wi.x, qb = wi.y, sub0 = wi.w & 0xffff, nq = (wi.w >> 16) & 0xff;
-      const bool split = (wi.w >> 24) != 0;
-      const int n_kv = wi.z * g.n_sub;
+      const bool split = ((wi.w >> 24) & 1) != 0;
+      const bool textq = ((wi.w >> 25) & 1) != 0;
+      const int n_vid = wi.z * g.n_sub;          // video key slabs, then the text slabs (always 128 wide)
+      const int n_kv = n_vid + g.n_ts;
       const bool use_o1 = (nq > 1) || (split && n_kv > 1);
       const bool active = (qi == 0) || use_o1;
       float m_ref = neg_inf;  // running reference maximum, scaled log2 domain
@@ -1021,7 +1053,7 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
         const int r_last = g.n_sub - 1;
         int rj = (j0 > r_last) ? 0 : j0;   // j mod n_sub, carried along (no division in the loop)
         for (int j = j0; ok && j < n_kv; j += dj) {
-          const int nk = (rj == r_last) ? g.n_last : kSlabTokens;
+          const int nk = (rj == r_last && j < n_vid) ? g.n_last : kSlabTokens;
           rj = (rj == r_last) ? 0 : rj + 1;
           if (dj == 2) rj = (rj == r_last) ? 0 : rj + 1;
           ok = mbar_wait_warp(bar(kBarSFull + qi), cnt_s & 1u, abort_flag, 0x300 + qi);
@@ -1128,14 +1160,18 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
       mbar_arrive(bar(kBarOEmpty + qi));
       if (split && use_o1) mbar_arrive(bar(kBarOEmpty + 1));
       int t0, h0, w0, et, eh, ew, ntok, last;
-      slab_origin(g, qb, sub0 + qi, t0, h0, w0);
-      slab_shape(g, sub0 + qi, et, eh, ew, ntok, last);
-      {
+      const float lse_row = empty ? neg_inf : (m_ref + log2f(l)) * 0.6931471805599453f;
+      if (textq) {   // text slab: rows are consecutive text tokens; they follow the L video tokens
+        t0 = 0; h0 = 0; w0 = (sub0 + qi) * kSlabTokens; last = 2;
+        if (w0 + row < g.n_text) prm.lse[(long long)head * g.Lt + g.L + w0 + row] = lse_row;
+      } else {
+        slab_origin(g, qb, sub0 + qi, t0, h0, w0);
+        slab_shape(g, sub0 + qi, et, eh, ew, ntok, last);
         const int wi_ = row % ew, hi_ = (row / ew) % eh, ti_ = row / (ew * eh);
         const int t = t0 + ti_, hh = h0 + hi_, ww = w0 + wi_;
         if (row < ntok && t < g.T && hh < g.H && ww < g.W) {
           const long long tok = ((long long)t * g.H + hh) * g.W + ww;
-          prm.lse[(long long)head * g.L + tok] = empty ? neg_inf : (m_ref + log2f(l)) * 0.6931471805599453f;
+          prm.lse[(long long)head * g.Lt + tok] = lse_row;
         }
       }
       fence_async_smem();

@@ -27,6 +27,12 @@ struct Geom {
   int items_per_block;     // work items per query block = ceil(n_sub / 2)
   float scale_log2;        // softmax scale times log2(e)
   long long L;             // T*H*W
+  // joint video + text sequences: n_text text tokens follow the L video tokens of every head
+  int n_text;              // 0: video only
+  int n_ts;                // text slabs of 128 tokens = ceil(n_text / 128)
+  int n_titems;            // work items of the text queries per head = ceil(n_ts / 2)
+  int items_per_head;      // NB * items_per_block + n_titems
+  long long Lt;            // L + n_text: tokens per head, row length of lse
 };
 
 struct HeadParamsArray {
@@ -35,7 +41,7 @@ struct HeadParamsArray {
 
 // One unit of work of the attention kernel: up to two query slabs of one query block.
 // x = head, y = query block id, z = number of attended key blocks,
-// w = first slab index | (number of slabs << 16)
+// w = first slab index | (number of slabs << 16) | (split-KV mode << 24) | (text-query item << 25)
 typedef int4 WorkItem;
 
 // Layout of the per-device workspace (all int32 words).

@@ -19,7 +19,7 @@ cudaError_t launch_mask_build(const HeadParamsArray& hp, const int* head_bases, 
 cudaError_t launch_plan(const HeadParamsArray& hp, const Geom& g, int head0, int n_heads_here, int* ws_header,
                         psa_head_params* hp_dev, WorkItem* items, cudaStream_t stream);
 struct TensorMaps {
-  CUtensorMap q[2], k[2], v[2], o[2];  // [0]: full 128-token slab box, [1]: a block's last slab
+  CUtensorMap q[3], k[3], v[3], o[3];  // [0]: full 128-token slab box, [1]: a block's last slab, [2]: text slab
 };
 cudaError_t launch_attn(const TensorMaps& tm, const Geom& g, const WorkItem* items, const psa_head_params* hp_dev,
                         int* ws_header, float* lse, int n_items, int n_sms, bool shared_qkv, cudaStream_t stream);
@@ -122,6 +122,20 @@ int make_geom(const psa_problem* prob, int T, int H, int W, bool for_attn, Geom*
     g->items_per_block = (n_sub + 1) / 2;
     g->scale_log2 = prob->scale * 1.4426950408889634f;
   }
+  g->items_per_head = g->NB * g->items_per_block;
+  g->Lt = L;
+  return PSA_OK;
+}
+
+// Adds n_text text tokens per head to an attention geometry.
+int set_text(Geom* g, long long n_text) {
+  if (n_text < 0 || g->L + n_text >= (1ll << 31)) return PSA_ERR_INVALID_ARG;
+  g->n_text = (int)n_text;
+  g->n_ts = (int)((n_text + kSlabTokens - 1) / kSlabTokens);
+  if (g->n_ts > 0xffff) return PSA_ERR_UNSUPPORTED;
+  g->n_titems = (g->n_ts + 1) / 2;
+  g->items_per_head = g->NB * g->items_per_block + g->n_titems;
+  g->Lt = g->L + n_text;
   return PSA_OK;
 }
 
@@ -181,6 +195,23 @@ int encode_map(CUtensorMap* tm, const void* base, const Geom& g, long long strid
   return r == CUDA_SUCCESS ? PSA_OK : PSA_ERR_INVALID_ARG;
 }
 
+// Map of the text tokens of every head: a [heads][n_text][128] view starting L tokens into each head,
+// box = 128 tokens x 64 columns (same shared-memory image as a full video slab).
+int encode_text_map(CUtensorMap* tm, const void* base, const Geom& g, long long stride_head, long long stride_token,
+                    int n_heads_here) {
+  const cuuint64_t st = (cuuint64_t)stride_token * 2;
+  const cuuint64_t dims[5] = {(cuuint64_t)kHeadDim, (cuuint64_t)g.n_text, 1, 1, (cuuint64_t)n_heads_here};
+  const cuuint64_t strides[4] = {st, st * g.n_text, st * g.n_text,
+                                 n_heads_here > 1 ? (cuuint64_t)stride_head * 2 : st * g.n_text};
+  const cuuint32_t box[5] = {64, (cuuint32_t)kSlabTokens, 1, 1, 1};
+  const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+  const void* text0 = static_cast<const uint16_t*>(base) + g.L * stride_token;
+  const CUresult r = g_encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(text0), dims, strides, box,
+                              estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? PSA_OK : PSA_ERR_INVALID_ARG;
+}
+
 // Strides (in elements) of the inputs and of the output of one attention launch.
 struct Layout {
   long long in_head, in_token;    // q, k, v
@@ -198,6 +229,14 @@ int encode_maps(TensorMaps* tm, const void* q, const void* k, const void* v, voi
     if ((rc = encode_map(&tm->k[last], k, g, lay.in_head, lay.in_token, n_in, last != 0)) != PSA_OK) return rc;
     if ((rc = encode_map(&tm->v[last], v, g, lay.in_head, lay.in_token, n_in, last != 0)) != PSA_OK) return rc;
     if ((rc = encode_map(&tm->o[last], out, g, lay.out_head, lay.out_token, n_heads_here, last != 0)) != PSA_OK) return rc;
+  }
+  if (g.n_text > 0) {
+    if ((rc = encode_text_map(&tm->q[2], q, g, lay.in_head, lay.in_token, n_in)) != PSA_OK) return rc;
+    if ((rc = encode_text_map(&tm->k[2], k, g, lay.in_head, lay.in_token, n_in)) != PSA_OK) return rc;
+    if ((rc = encode_text_map(&tm->v[2], v, g, lay.in_head, lay.in_token, n_in)) != PSA_OK) return rc;
+    if ((rc = encode_text_map(&tm->o[2], out, g, lay.out_head, lay.out_token, n_heads_here)) != PSA_OK) return rc;
+  } else {  // never used; keep the descriptors valid
+    tm->q[2] = tm->q[0]; tm->k[2] = tm->k[0]; tm->v[2] = tm->v[0]; tm->o[2] = tm->o[0];
   }
   return PSA_OK;
 }
@@ -350,7 +389,7 @@ static int run_attn(const void* q, const void* k, const void* v, void* out, floa
   rc = load_driver_entry();
   if (rc != PSA_OK) return rc;
   const int chunk = n_heads < kMaxHeads ? n_heads : kMaxHeads;
-  const size_t items_bytes = sizeof(WorkItem) * (size_t)chunk * g.NB * g.items_per_block;
+  const size_t items_bytes = sizeof(WorkItem) * (size_t)chunk * g.items_per_head;
   const size_t hp_off = sizeof(int) * kWsHeaderWords;
   const size_t items_off = (hp_off + sizeof(psa_head_params) * kMaxHeads + 255) & ~size_t(255);
   rc = ensure_workspace(ws, items_off + items_bytes);
@@ -373,9 +412,9 @@ static int run_attn(const void* q, const void* k, const void* v, void* out, floa
     gh.n_heads = n_here;
     if (launch_plan(hp, gh, 0, n_here, ws_header, hp_dev, items, st) != cudaSuccess) return PSA_ERR_CUDA;
     ++g_launches;
-    const int n_items = n_here * g.NB * g.items_per_block;
+    const int n_items = n_here * g.items_per_head;
     if (g_ev_start && g_ev_stop) cudaEventRecord(g_ev_start, st);
-    if (launch_attn(tm, gh, items, hp_dev, ws_header, lse + (long long)head0 * g.L, n_items, ws->n_sms, lay.shared_qkv, st) !=
+    if (launch_attn(tm, gh, items, hp_dev, ws_header, lse + (long long)head0 * g.Lt, n_items, ws->n_sms, lay.shared_qkv, st) !=
         cudaSuccess)
       return PSA_ERR_CUDA;
     if (g_ev_start && g_ev_stop) cudaEventRecord(g_ev_stop, st);
@@ -450,6 +489,26 @@ int psa_attn_fwd_batched(const void* q, const void* k, const void* v, void* out,
   return PSA_OK;
 }
 
+int psa_attn_fwd_joint(const void* q, const void* k, const void* v, void* out, float* lse,
+                       const psa_head_params* head_params, const psa_problem* prob, int64_t n_text, int T, int H, int W,
+                       void* stream) {
+  Geom g;
+  int rc = make_geom(prob, T, H, W, true, &g);
+  if (rc != PSA_OK) return rc;
+  if ((rc = set_text(&g, n_text)) != PSA_OK) return rc;
+  if (!q || !k || !v || !out || !lse || !head_params) return PSA_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || (reinterpret_cast<uintptr_t>(lse) & 3u))
+    return PSA_ERR_INVALID_ARG;
+  if (out == q || out == k || out == v) return PSA_ERR_INVALID_ARG;
+  if (prob->stride_token < kHeadDim || (prob->stride_token % 8) != 0) return PSA_ERR_INVALID_ARG;
+  if (prob->n_heads > 1 && (prob->stride_head < kHeadDim || (prob->stride_head % 8) != 0)) return PSA_ERR_INVALID_ARG;
+  for (int h = 0; h < prob->n_heads; ++h)
+    if (!valid_params(head_params[h])) return PSA_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lock(g_mu);
+  const Layout lay = {prob->stride_head, prob->stride_token, prob->stride_head, prob->stride_token, false};
+  return run_attn(q, k, v, out, lse, head_params, prob->n_heads, g, lay, static_cast<cudaStream_t>(stream));
+}
+
 // ---- PSA-Search for one head (Algorithm 3) ------------------------------------------------------
 // scratch layout: outputs of the n_cand candidates and of full attention ((n_cand + 1) x L x 128 bf16),
 // their lse ((n_cand + 1) x L fp32), the partial sums of the loss reduction.
@@ -521,7 +580,7 @@ int psa_attn_fwd_noalloc(const void* q, const void* k, const void* v, void* out,
   for (int h = 0; h < prob->n_heads; ++h)
     if (!valid_params(head_params[h])) return PSA_ERR_INVALID_ARG;
   // the fixed scratch bounds the problem: one launch worth of heads and kNoAllocMaxItems items
-  const long long n_items_ll = (long long)prob->n_heads * g.NB * g.items_per_block;
+  const long long n_items_ll = (long long)prob->n_heads * g.items_per_head;
   if (prob->n_heads > kMaxHeads || n_items_ll > kNoAllocMaxItems) return PSA_ERR_CAPACITY;
 
   std::lock_guard<std::mutex> lock(g_mu);
