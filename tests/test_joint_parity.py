@@ -88,3 +88,32 @@ def test_zero_text_tokens_is_the_video_only_call_bit_for_bit(B):
     o1, l1 = B.psa_attn_fwd(q, k, v, params, grid, tile, SCALE)
     o2, l2 = B.psa_attn_fwd_joint(q, k, v, params, grid, tile, SCALE, 0)
     assert torch.equal(o1.view(torch.int16), o2.view(torch.int16)) and torch.equal(l1, l2)
+
+
+def test_hunyuan_768p_with_256_text_tokens_sampled_rows(B):
+    """Full-size joint call (the launch configuration of the timings): HunyuanVideo 768p shape plus 256
+    text tokens; four heads are generated and run, sampled video rows, a whole edge brick and sampled text
+    rows of each are compared with the oracle against all keys."""
+    w = WL.workload("hunyuan_768p")
+    grid, tile, nt = w["grid"], w["tile"], 256
+    T, H, W = grid
+    L = T * H * W
+    heads = [0, 7, 14, 23]
+    params = [tuple(w["head_params"][h]) for h in heads]
+    bits = {n: np.stack([WL.head_bits(w["seed"], n, h, L + nt) for h in heads]) for n in ("q", "k", "v")}
+    q, k, v = (_to_dev(bits[n]) for n in ("q", "k", "v"))
+    out, lse = B.psa_attn_fwd_joint(q, k, v, params, grid, tile, SCALE, nt)
+    st, detail = B.psa_last_device_status()
+    assert st == 0, (st, hex(detail))
+    out_h, lse_h = _bf16_to_f64(out), lse.cpu().numpy().astype(np.float64)
+    for i, hd in enumerate(heads):
+        rows = set(WL.sample_rows(w["seed"], hd, L, 24))
+        rows |= {L + r for r in WL.sample_rows(w["seed"] + 1, hd, nt, 12)} | {L, L + nt - 1}
+        bt, bh, bw = tile     # the last brick of the grid
+        rows |= {(t * H + h) * W + x for t in range(T - bt, T) for h in range(H - bh, H) for x in range(W - bw, W) if (h + x) % 4 == 0}
+        rows = sorted(rows)
+        qf, kf, vf = (O.bf16_bits_to_f64(bits[n][i]) for n in ("q", "k", "v"))
+        ro, rl = O.attention_rows_with_text(qf, kf, vf, rows, params[i], T, H, W, tuple(tile), SCALE, nt)
+        err = np.abs(out_h[i][rows] - ro)
+        assert err.max() <= OUT_MAX and err.mean() <= OUT_MEAN, (hd, err.max(), err.mean())
+        assert np.abs(lse_h[i][rows] - rl).max() <= LSE_MAX, hd

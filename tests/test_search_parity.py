@@ -133,3 +133,26 @@ def test_select_matches_oracle_and_hand_examples(B):
         assert B.psa_search_select_at_sparsity(ls, sp, target) == O.search_select_at_sparsity(ls, sp, target)
     with pytest.raises(ValueError):
         B.psa_search_select([0.1], [0.1, 0.2], 0.5)
+
+
+@pytest.mark.gpu
+def test_losses_at_full_size_agree_with_the_attention_entry_point(B):
+    """At the 75,600-token shape the oracle cannot form the dense reference; here the device reduction is
+    checked against the mean squared difference of outputs computed by separate psa_attn_fwd calls (whose
+    parity with the oracle is tested on sampled rows elsewhere).  Same kernels, different plumbing: shared
+    q/k/v maps, candidate batching, scratch layout and the two-stage reduction are what is under test."""
+    w = WL.workload("wan14b_720p")
+    grid, tile = w["grid"], w["tile"]
+    T, H, W = grid
+    L = T * H * W
+    cands = [tuple(w["head_params"][h]) for h in (0, 2, 12)]
+    bits = {n: WL.head_bits(w["seed"], n, 3, L) for n in ("q", "k", "v")}
+    q, k, v = (_to_dev(bits[n]) for n in ("q", "k", "v"))
+    got = B.psa_search_losses(q, k, v, cands, grid, tile, SCALE).cpu().numpy().astype(np.float64)
+    assert B.psa_last_device_status()[0] == 0
+    Tp, Hp, Wp = O.block_grid(T, H, W, tuple(tile))
+    full, _ = B.psa_attn_fwd(q[None], k[None], v[None], [(Tp, 0, INF, Hp * Wp, 0, INF)], grid, tile, SCALE)
+    for c, p in enumerate(cands):
+        o, _ = B.psa_attn_fwd(q[None], k[None], v[None], [p], grid, tile, SCALE)
+        ref = float(((o.double() - full.double()) ** 2).mean())
+        assert abs(got[c] - ref) <= 1e-6 * ref + 1e-12, (c, got[c], ref)
