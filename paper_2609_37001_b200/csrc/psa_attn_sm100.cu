@@ -805,7 +805,10 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
   } else if (warp == kWarpMma) {
     // ======================================================================= MMA warp
     constexpr uint32_t kIdescPV = instr_desc(true, 128);  // N = head_dim
-    uint32_t tile_g = 0, pair_g = 0;
+    // ring slot of the next tile and pair barrier of the next arrival: wrapping index + phase bit
+    uint32_t slot_i = 0, pair_i = 0, pair_ph = 0;
+    auto slot_next = [&](uint32_t sl) -> uint32_t { return sl + 1u == (uint32_t)kNumSlots ? 0u : sl + 1u; };
+    auto pair_adv = [&]() { if (++pair_i == (uint32_t)kNumPairBars) { pair_i = 0; pair_ph ^= 1u; } };
     uint32_t it_q0 = 0, it_q1 = 0;
     uint32_t cnt_s0 = 0, cnt_s1 = 0;  // P_i tiles consumed so far
     bool ok = true;
@@ -884,11 +887,11 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
         // Ring order (see the load warp): K_0, K_1, (V_0, K_2), (V_1, K_3), ..., V_{n-2}, V_{n-1}.
         int r0 = 0;   // residue of the slab whose scores are issued next
         for (int j = 0; ok && j < 2 && j < n_kv; ++j) {
-          ok = mbar_wait_warp(bar(kBarPairFull + pair_g % kNumPairBars), (pair_g / kNumPairBars) & 1u, abort_flag, 0x230);
+          ok = mbar_wait_warp(bar(kBarPairFull + pair_i), pair_ph, abort_flag, 0x230);
           if (!ok) break;
-          ++pair_g;
-          const uint32_t slot = tile_g % kNumSlots;
-          ++tile_g;
+          pair_adv();
+          const uint32_t slot = slot_i;
+          slot_i = slot_next(slot_i);
           tc_fence_after();
           if (elect_one()) {
             issue_qk(0, slot, nk_j(j, r0), j);
@@ -902,14 +905,13 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
         for (int j = 0; ok && j < n_kv; ++j) {
           const int i = j & 1;
           const uint32_t cs = i == 0 ? cnt_s0 : cnt_s1;
-          ok = mbar_wait2_warp(bar(kBarPairFull + pair_g % kNumPairBars), (pair_g / kNumPairBars) & 1u,
-                               bar(kBarPHalf + i), cs & 1u, abort_flag, 0x231, 0x234 + i);
+          ok = mbar_wait2_warp(bar(kBarPairFull + pair_i), pair_ph, bar(kBarPHalf + i), cs & 1u, abort_flag, 0x231, 0x234 + i);
           if (!ok) break;
-          ++pair_g;
+          pair_adv();
           const bool more = (j + 2 < n_kv);
-          const uint32_t vslot = tile_g % kNumSlots;
-          const uint32_t kslot = (tile_g + 1) % kNumSlots;
-          tile_g += more ? 2u : 1u;
+          const uint32_t vslot = slot_i;
+          const uint32_t kslot = slot_next(slot_i);
+          slot_i = more ? slot_next(kslot) : kslot;
           const int nk_cur = nk_j(j, rj);
           rj = r_inc(rj);
           tc_fence_after();
@@ -934,79 +936,96 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
         }
         if (!ok) break;
       } else if (n_kv > 0) {
-        // first key slab: both S tiles
+        // first key slab: both S tiles (a two-slab item: nq == 2)
         {
-          ok = mbar_wait_warp(bar(kBarPairFull + pair_g % kNumPairBars), (pair_g / kNumPairBars) & 1u, abort_flag, 0x210);
+          ok = mbar_wait_warp(bar(kBarPairFull + pair_i), pair_ph, abort_flag, 0x210);
           if (!ok) break;
-          ++pair_g;
-          const uint32_t slot = tile_g % kNumSlots;
-          ++tile_g;
+          pair_adv();
+          const uint32_t slot = slot_i;
+          slot_i = slot_next(slot_i);
           tc_fence_after();
           if (elect_one()) {
-#pragma unroll
-            for (int i = 0; i < 2; ++i) {
-              if (i < nq) {
-                issue_qk(i, slot, nk_j(0, 0), i);
-                tc_commit(bar(kBarSFull + i));
-              }
-            }
+            issue_qk(0, slot, nk_j(0, 0), 0);
+            tc_commit(bar(kBarSFull + 0));
+            issue_qk(1, slot, nk_j(0, 0), 1);
+            tc_commit(bar(kBarSFull + 1));
             tc_commit(bar(kBarSlotEmpty + slot));
           }
           __syncwarp();
         }
+        // Per key slab j: P_0's first half -> P V (4 MMAs); all of P_0 -> the other 4 + next scores of
+        // tile 0; the same for tile 1.  The barrier of V_j / K_{j+1} (loaded long before) is waited for
+        // together with another wait, never on its own, and the bookkeeping for the next slab runs
+        // while the queued MMAs drain.
         int rj = 0;
+        bool pair_seen = false;   // V_j / K_{j+1} already known to have arrived
         for (int j = 0; ok && j < n_kv; ++j) {
           const int nk_cur = nk_j(j, rj);
           rj = r_inc(rj);
           const int nk_next = nk_j(j + 1, rj);
-          // V_j and (unless this is the last slab) K_{j+1} arrive under one barrier; it is waited
-          // for together with the first half of P_0 (one shared-memory round trip for both)
           TRACE(2, j, 5);
           const bool more = (j + 1 < n_kv);
-          const uint32_t vslot = tile_g % kNumSlots;
-          const uint32_t kslot = (tile_g + 1) % kNumSlots;
-          tile_g += more ? 2u : 1u;
-          ok = mbar_wait2_warp(bar(kBarPairFull + pair_g % kNumPairBars), (pair_g / kNumPairBars) & 1u,
-                               bar(kBarPHalf + 0), cnt_s0 & 1u, abort_flag, 0x211, 0x224);
+          const uint32_t vslot = slot_i;
+          const uint32_t kslot = slot_next(slot_i);
+          slot_i = more ? slot_next(kslot) : kslot;
+          if (pair_seen) ok = mbar_wait_warp(bar(kBarPHalf + 0), cnt_s0 & 1u, abort_flag, 0x224);
+          else ok = mbar_wait2_warp(bar(kBarPairFull + pair_i), pair_ph, bar(kBarPHalf + 0), cnt_s0 & 1u, abort_flag, 0x211, 0x224);
           if (!ok) break;
+          pair_adv();
           TRACE(2, j, 3);
-          ++pair_g;
+          tc_fence_after();
+          TRACE(2, j, 0);
+          if (elect_one()) issue_pv_half(0, vslot, 0, j > 0, nk_cur);
           bool half1_done = false;   // first half of P_1 already seen complete
-#pragma unroll
-          for (int i = 0; i < 2; ++i) {
-            if (!ok || i >= nq) break;
-            const uint32_t cs = i == 0 ? cnt_s0 : cnt_s1;
-            if (i == 1 && !half1_done) {
-              ok = mbar_wait_warp(bar(kBarPHalf + 1), cs & 1u, abort_flag, 0x225);
-              if (!ok) break;
-            }
-            tc_fence_after();
-            TRACE(2 + i, j, 0);
-            if (elect_one()) issue_pv_half(i, vslot, 0, j > 0, nk_cur);
-            if (i == 0 && nq > 1) {
-              ok = mbar_wait_probe_warp(bar(kBarPReady + 0), cs & 1u, bar(kBarPHalf + 1), cnt_s1 & 1u, abort_flag,
-                                        0x220, &half1_done);
+          ok = mbar_wait_probe_warp(bar(kBarPReady + 0), cnt_s0 & 1u, bar(kBarPHalf + 1), cnt_s1 & 1u, abort_flag, 0x220,
+                                    &half1_done);
+          if (!ok) break;
+          ++cnt_s0;
+          tc_fence_after();
+          TRACE(2, j, 1);
+          if (elect_one()) {
+            issue_pv_half(0, vslot, 1, true, nk_cur);
+            if (more) {
+              issue_qk(0, kslot, nk_next, 0);
+              tc_commit(bar(kBarSFull + 0));
             } else {
-              ok = mbar_wait_warp(bar(kBarPReady + i), cs & 1u, abort_flag, 0x220 + i);
+              tc_commit(bar(kBarOFull + 0));
             }
-            if (!ok) break;
-            if (i == 0) ++cnt_s0; else ++cnt_s1;
-            tc_fence_after();
-            TRACE(2 + i, j, 1);
-            if (elect_one()) {
-              issue_pv_half(i, vslot, 1, true, nk_cur);
-              if (i == nq - 1) tc_commit(bar(kBarSlotEmpty + vslot));
-              if (more) {
-                issue_qk(i, kslot, nk_next, i);
-                tc_commit(bar(kBarSFull + i));
-                if (i == nq - 1) tc_commit(bar(kBarSlotEmpty + kslot));
-              } else {
-                tc_commit(bar(kBarOFull + i));
-              }
-            }
-            __syncwarp();
-            TRACE(2 + i, j, 2);
           }
+          __syncwarp();
+          TRACE(2, j, 2);
+          if (!half1_done) {
+            ok = mbar_wait_warp(bar(kBarPHalf + 1), cnt_s1 & 1u, abort_flag, 0x225);
+            if (!ok) break;
+          }
+          tc_fence_after();
+          TRACE(3, j, 0);
+          if (elect_one()) issue_pv_half(1, vslot, 0, j > 0, nk_cur);
+          // all of P_1, and (one round trip) the loads of the next slab
+          pair_seen = false;
+          if (more) {
+            ok = mbar_wait_probe_warp(bar(kBarPReady + 1), cnt_s1 & 1u, bar(kBarPairFull + pair_i), pair_ph, abort_flag, 0x221,
+                                      &pair_seen);
+          } else {
+            ok = mbar_wait_warp(bar(kBarPReady + 1), cnt_s1 & 1u, abort_flag, 0x221);
+          }
+          if (!ok) break;
+          ++cnt_s1;
+          tc_fence_after();
+          TRACE(3, j, 1);
+          if (elect_one()) {
+            issue_pv_half(1, vslot, 1, true, nk_cur);
+            tc_commit(bar(kBarSlotEmpty + vslot));
+            if (more) {
+              issue_qk(1, kslot, nk_next, 1);
+              tc_commit(bar(kBarSFull + 1));
+              tc_commit(bar(kBarSlotEmpty + kslot));
+            } else {
+              tc_commit(bar(kBarOFull + 1));
+            }
+          }
+          __syncwarp();
+          TRACE(3, j, 2);
         }
         if (!ok) break;
       } else {
