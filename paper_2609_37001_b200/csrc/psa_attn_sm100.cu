@@ -22,8 +22,8 @@
 // P_i overwrite the first columns of S_i.  A key slab has 128 keys, or 112/96/64 for the last
 // slab of a block whose token count is not a multiple of 128.
 // Every wait is bounded; on expiry the CTA records a status word and unwinds.
-// Build-time knobs: PSA_EMU_PAIRS (share of exponentials computed by a polynomial on the FMA
-// pipe, default 0), PSA_TRACE (cycle stamps).
+// Build-time knob: PSA_EMU_PAIRS (share of exponentials computed by a polynomial on the FMA
+// pipe, default 0).
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -44,7 +44,10 @@ constexpr unsigned long long kTimeoutNs = 2000000000ull;
 constexpr uint32_t kOffQ = 0;                                   // 2 slabs
 constexpr uint32_t kOffRing = 2 * kSlabBytes;                   // kNumSlots slabs
 constexpr uint32_t kOffBar = kOffRing + kNumSlots * kSlabBytes; // mbarriers
-constexpr int kNumPairBars = 3;
+// One load barrier per ring slot: a barrier is armed again only after as many further tiles as
+// there are slots have been issued, i.e. after the tiles of its previous phase were consumed
+// (tiles that travel alone -- the first K and the last V of an item -- each take a barrier).
+constexpr int kNumPairBars = kNumSlots;
 constexpr int kBarQFull = 0, kBarQEmpty = 2, kBarPairFull = 4, kBarSlotEmpty = kBarPairFull + kNumPairBars,
               kBarSFull = kBarSlotEmpty + kNumSlots, kBarPHalf = kBarSFull + 2, kBarPReady = kBarPHalf + 2,
               kBarOFull = kBarPReady + 2, kBarOEmpty = kBarOFull + 2, kBarSchedFull = kBarOEmpty + 2,
@@ -303,21 +306,6 @@ __device__ __forceinline__ bool elect_one() {
   return pred != 0;
 }
 
-// Developer knob (-DPSA_TRACE): CTA 0 records cycle stamps of its second work item.
-#ifdef PSA_TRACE
-__device__ long long g_trace[4 * 64 * 8];
-__device__ long long g_trace_items[2 * 256 * 4];
-__device__ long long g_trace_w[8 * 64 * 2];
-#define TRACE(role, j, k)                                                                     \
-  do {                                                                                          \
-    if (blockIdx.x == 0 && n == 1 && (j) < 64 && (threadIdx.x & 31) == 0 &&                     \
-        ((threadIdx.x >> 5) & 3) == (((role) < 2 ? kFirstSoftmaxWarp : kWarpMma) & 3))         \
-      g_trace[((role) * 64 + (j)) * 8 + (k)] = clock64();                                       \
-  } while (0)
-#else
-#define TRACE(role, j, k) do { } while (0)
-#endif
-
 // ----------------------------------------------------------------------------- planning
 // Work order: per head, query blocks ranked by attended key-block count (largest first),
 // heads kept together so that concurrently running CTAs share K/V in L2.
@@ -428,12 +416,7 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t lo) { return ((uint64_t)k
 template <int NK>
 __device__ __forceinline__ void softmax_slab(uint32_t tS, uint32_t tO, const uint4 meta, bool first,
                                              float scale_log2, float& m_ref, float& l, uint32_t bar_half,
-                                             uint32_t bar_ready, long long* tr = nullptr) {
-#ifdef PSA_TRACE
-#define STAMP(k) do { if (tr) tr[k] = clock64(); } while (0)
-#else
-#define STAMP(k) do { } while (0)
-#endif
+                                             uint32_t bar_ready) {
   constexpr int NFULL = NK / 32, REM = NK % 32;
   static_assert(NK % 16 == 0 && NK >= 64 && NK <= 128 && (REM == 0 || REM == 16), "unsupported slab width");
   const float neg_inf = __int_as_float(0xff800000);
@@ -442,14 +425,12 @@ __device__ __forceinline__ void softmax_slab(uint32_t tS, uint32_t tO, const uin
   for (int c4 = 0; c4 < NFULL; ++c4) tc_ld32(tS + c4 * 32, s + c4 * 32);
   if (REM) tc_ld16(tS + NFULL * 32, s + NFULL * 32);
   tc_wait_ld();
-  STAMP(1);
   if ((meta.x & meta.y & meta.z & meta.w) != 0xffffffffu) {  // 3D-padding: padded key positions score -inf
     const uint32_t v[4] = {meta.x, meta.y, meta.z, meta.w};
 #pragma unroll
     for (int c = 0; c < NK; ++c)
       if (!((v[c >> 5] >> (c & 31)) & 1u)) s[c] = 0xff800000u;
   }
-  STAMP(7);
   // eight independent chains (NK is a multiple of 16): shorter dependency depth
   float a[8];
 #pragma unroll
@@ -483,7 +464,6 @@ __device__ __forceinline__ void softmax_slab(uint32_t tS, uint32_t tO, const uin
     }
   }
   const float m_use = (m_ref == neg_inf) ? 0.f : m_ref;
-  STAMP(2);
   const uint64_t sc2 = pack2(scale_log2, scale_log2), negm2 = pack2(-m_use, -m_use);
   uint64_t sum2 = pack2(0.f, 0.f);
   // probabilities exp2(scale*s - m_use), bf16, written over the scores in chunks of 32 keys
@@ -511,11 +491,9 @@ __device__ __forceinline__ void softmax_slab(uint32_t tS, uint32_t tO, const uin
     exp_chunk(c4 * 32, 16, pk);
     tc_st16(tS + c4 * 16, pk);
     if (c4 == 1) {  // the first 64 keys are final: their P V MMAs may start
-      STAMP(5);
       tc_wait_st();
       tc_fence_before();
       mbar_arrive(bar_half);
-      STAMP(3);
     }
   }
   if (REM) {
@@ -526,11 +504,9 @@ __device__ __forceinline__ void softmax_slab(uint32_t tS, uint32_t tO, const uin
   float sum0, sum1;
   unpack2(sum2, sum0, sum1);
   l += sum0 + sum1;
-  STAMP(6);
   tc_wait_st();
   tc_fence_before();
   mbar_arrive(bar_ready);
-#undef STAMP
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -858,12 +834,6 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
       const int n_vid = wi.z * g.n_sub;          // video key slabs, then the text slabs (always 128 wide)
       const int n_kv = n_vid + g.n_ts;
       auto nk_j = [&](int j, int r) -> int { return j >= n_vid ? kSlabTokens : nk_at(r); };
-#ifdef PSA_TRACE
-      if ((blockIdx.x == 0 || blockIdx.x == 77) && n < 256 && lane == 0) {
-        long long* r = g_trace_items + ((blockIdx.x == 0 ? 0 : 1) * 256 + n) * 4;
-        r[0] = clock64(); r[1] = n_kv; r[2] = wi.x; r[3] = (long long)globaltimer_ns();
-      }
-#endif
       // which accumulators this item uses: both for a two-slab item, and for a split-KV item
       // with at least two key slabs (even slabs -> O_0, odd slabs -> O_1)
       const bool use_o1 = (nq > 1) || (split && n_kv > 1);
@@ -963,7 +933,6 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
           const int nk_cur = nk_j(j, rj);
           rj = r_inc(rj);
           const int nk_next = nk_j(j + 1, rj);
-          TRACE(2, j, 5);
           const bool more = (j + 1 < n_kv);
           const uint32_t vslot = slot_i;
           const uint32_t kslot = slot_next(slot_i);
@@ -972,9 +941,7 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
           else ok = mbar_wait2_warp(bar(kBarPairFull + pair_i), pair_ph, bar(kBarPHalf + 0), cnt_s0 & 1u, abort_flag, 0x211, 0x224);
           if (!ok) break;
           pair_adv();
-          TRACE(2, j, 3);
           tc_fence_after();
-          TRACE(2, j, 0);
           if (elect_one()) issue_pv_half(0, vslot, 0, j > 0, nk_cur);
           bool half1_done = false;   // first half of P_1 already seen complete
           ok = mbar_wait_probe_warp(bar(kBarPReady + 0), cnt_s0 & 1u, bar(kBarPHalf + 1), cnt_s1 & 1u, abort_flag, 0x220,
@@ -982,7 +949,6 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
           if (!ok) break;
           ++cnt_s0;
           tc_fence_after();
-          TRACE(2, j, 1);
           if (elect_one()) {
             issue_pv_half(0, vslot, 1, true, nk_cur);
             if (more) {
@@ -993,13 +959,11 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
             }
           }
           __syncwarp();
-          TRACE(2, j, 2);
           if (!half1_done) {
             ok = mbar_wait_warp(bar(kBarPHalf + 1), cnt_s1 & 1u, abort_flag, 0x225);
             if (!ok) break;
           }
           tc_fence_after();
-          TRACE(3, j, 0);
           if (elect_one()) issue_pv_half(1, vslot, 0, j > 0, nk_cur);
           // all of P_1, and (one round trip) the loads of the next slab
           pair_seen = false;
@@ -1012,7 +976,6 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
           if (!ok) break;
           ++cnt_s1;
           tc_fence_after();
-          TRACE(3, j, 1);
           if (elect_one()) {
             issue_pv_half(1, vslot, 1, true, nk_cur);
             tc_commit(bar(kBarSlotEmpty + vslot));
@@ -1025,7 +988,6 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
             }
           }
           __syncwarp();
-          TRACE(3, j, 2);
         }
         if (!ok) break;
       } else {
@@ -1079,28 +1041,15 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
           if (!ok) break;
           ++cnt_s;
           tc_fence_after();
-          TRACE(qi, j, 0);
           // Read the slab's validity words first: shared memory is busy feeding the tensor core,
           // so the load's latency is overlapped with the TMEM loads that follow.
           const uint4 m = *reinterpret_cast<const uint4*>(meta + ((kv_g + (uint32_t)j) % kMetaRing) * 8);
           const uint32_t bh = bar(kBarPHalf + qi), br = bar(kBarPReady + qi);
-#ifdef PSA_TRACE
-          long long* tr = (blockIdx.x == 0 && n == 1 && j < 64 && (threadIdx.x & 127) == 0) ? g_trace + (qi * 64 + j) * 8 : nullptr;
-#else
-          long long* tr = nullptr;
-#endif
           const bool first = (j == j0);
-#ifdef PSA_TRACE
-          if (blockIdx.x == 0 && n == 1 && j < 64 && lane == 0) g_trace_w[((warp - kFirstSoftmaxWarp) * 64 + j) * 2] = clock64();
-#endif
-          if (nk == 128) softmax_slab<128>(tS, tO, m, first, g.scale_log2, m_ref, l, bh, br, tr);
-          else if (nk == 112) softmax_slab<112>(tS, tO, m, first, g.scale_log2, m_ref, l, bh, br, tr);
-          else if (nk == 96) softmax_slab<96>(tS, tO, m, first, g.scale_log2, m_ref, l, bh, br, tr);
-          else softmax_slab<64>(tS, tO, m, first, g.scale_log2, m_ref, l, bh, br, tr);
-          TRACE(qi, j, 4);
-#ifdef PSA_TRACE
-          if (blockIdx.x == 0 && n == 1 && j < 64 && lane == 0) g_trace_w[((warp - kFirstSoftmaxWarp) * 64 + j) * 2 + 1] = clock64();
-#endif
+          if (nk == 128) softmax_slab<128>(tS, tO, m, first, g.scale_log2, m_ref, l, bh, br);
+          else if (nk == 112) softmax_slab<112>(tS, tO, m, first, g.scale_log2, m_ref, l, bh, br);
+          else if (nk == 96) softmax_slab<96>(tS, tO, m, first, g.scale_log2, m_ref, l, bh, br);
+          else softmax_slab<64>(tS, tO, m, first, g.scale_log2, m_ref, l, bh, br);
         }
       }
       kv_g += (uint32_t)n_kv;
@@ -1278,15 +1227,3 @@ cudaError_t launch_attn(const TensorMaps& tm, const Geom& g, const WorkItem* ite
 
 }  // namespace psa
 
-
-#ifdef PSA_TRACE
-extern "C" int psa_debug_read_trace(long long* out, int n) {
-  return (int)cudaMemcpyFromSymbol(out, psa::g_trace, sizeof(long long) * n);
-}
-extern "C" int psa_debug_read_trace_w(long long* out, int n) {
-  return (int)cudaMemcpyFromSymbol(out, psa::g_trace_w, sizeof(long long) * n);
-}
-extern "C" int psa_debug_read_items(long long* out, int n) {
-  return (int)cudaMemcpyFromSymbol(out, psa::g_trace_items, sizeof(long long) * n);
-}
-#endif
