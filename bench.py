@@ -9,6 +9,10 @@ Wan 2.1 14B 720p (40 heads, 21x45x80 = 75,600 tokens, head_dim 128): psa_mask_bu
 kernel).  The metric is computed TFLOP/s: 4*d FLOP per attended real (query, key) pair
 divided by the time of a step.  N > 1 runs N independent replicas (the path has no
 exchange step); the value is the sum over replicas divided by the slowest replica's time.
+With --gpus N > 1 and no WORLD_SIZE in the environment the script starts the N ranks itself
+(one process per GPU, NCCL, loopback rendezvous); under torchrun it uses the ranks it is given.
+--ulysses times the head-sharded call on sequence-sharded inputs instead (two all-to-all
+re-layouts around the kernel, timed separately from it).
 
 Prints ONE JSON line (rank 0).  --impl reference times the fp64 CPU oracle on a bounded
 sample of the same workload on the host cores.
@@ -32,6 +36,10 @@ UNIT = "TFLOP/s"
 HEAD_DIM = 128
 SCALE = 1.0 / math.sqrt(128.0)
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+DATASHEET_BF16_TFLOPS = 2250.0   # nominal dense bf16 figure of the part (context beside the measured peak)
+# the other configurations of the benchmark set, timed at kernel level after the headline
+OTHER_CONFIGS = ["tiny", "wan13b_480p", "hunyuan_720p", "sweep_00", "sweep_25", "sweep_50", "sweep_75", "sweep_90",
+                 "ragged_75", "wan14b_720p_b3x8x16", "hunyuan_768p"]
 
 
 def load_peaks():
@@ -51,13 +59,40 @@ def workload_flops(w):
 
 
 def config_of(w, extra=None):
+    """Names the workload; identical in both arms (--impl ours / reference)."""
     T, H, W = w["grid"]
+    input_bytes = 3 * w["n_heads"] * T * H * W * HEAD_DIM * 2
     c = {"workload": w["name"], "grid": w["grid"], "tokens": T * H * W, "n_heads": w["n_heads"],
          "head_dim": HEAD_DIM, "mask_block": w["tile"], "tile_sparsity": w["tile_sparsity"],
-         "step": "psa_mask_build + psa_attn_fwd", "parallelism": "replicas"}
+         "step": "psa_mask_build + psa_attn_fwd", "parallelism": "replicas",
+         "l2_policy": ("inputs (%.1f GB) exceed L2; no flush needed" % (input_bytes / 1e9)) if input_bytes > 2.5e8
+                      else "inputs fit L2",
+         "peaks": load_peaks()["_source"]}
     if extra:
         c.update(extra)
     return c
+
+
+def slab_split(tile):
+    """(slabs per block, keys of the last slab) of a mask block, as the attention kernel splits it:
+    128-token slabs along the block's outermost axis of extent > 1, the last one possibly shorter."""
+    bt, bh, bw = tile
+    if bt > 1 or (bh == 1 and bw == 1):
+        extent, other = bt, bh * bw
+    elif bh > 1:
+        extent, other = bh, bt * bw
+    else:
+        extent, other = bw, bt * bh
+    c0 = 128 // other
+    n_sub = -(-extent // c0)
+    return n_sub, (extent - (n_sub - 1) * c0) * other
+
+
+def issued_flops(nnz, tile):
+    """FLOPs the tensor cores are asked for: every attended block pair costs (128 rows per query
+    slab) x (keys of every key slab) x 4 x head_dim, padded and idle rows included."""
+    n_sub, n_last = slab_split(tile)
+    return 4.0 * HEAD_DIM * nnz * (128.0 * n_sub) * (128.0 * (n_sub - 1) + n_last)
 
 
 # ----------------------------------------------------------------------------- CPU oracle leg
@@ -108,7 +143,7 @@ def run_reference(args, w):
     total = sum(times)
     value = 4.0 * HEAD_DIM * pairs / total / 1e12
     sample = f"per step: 16 seeded query rows of 1 head against all {w['grid'][0] * w['grid'][1] * w['grid'][2]} keys (incl. input generation and bf16->fp64 conversion)"
-    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "gpus_used": 0, "ranks_that_ran": 1,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / max(len(times), 1),
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": config_of(w),
@@ -219,24 +254,44 @@ def run_ours(args, w):
         if st != 0:
             raise SystemExit(f"device status {st} detail {hex(detail)}")
 
+        # ---- same-process calibration (harness only, outside the timed region): a bf16 torch.matmul
+        # exposes the clock state of this GPU at this moment next to the recorded peak
+        calib = None
+        if rank == 0 and not args.quick:
+            a = torch.randn((8192, 8192), device=dev, dtype=torch.bfloat16)
+            b = torch.randn((8192, 8192), device=dev, dtype=torch.bfloat16)
+            c = torch.empty_like(a)
+            best = float("inf")
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            for _ in range(8):
+                e0.record(stream)
+                torch.matmul(a, b, out=c)
+                e1.record(stream)
+                torch.cuda.synchronize()
+                best = min(best, e0.elapsed_time(e1))
+            calib = {"bf16_matmul_8192_tflops_best_of_8": 2.0 * 8192 ** 3 / (best * 1e-3) / 1e12,
+                     "recorded_peak_tflops": peaks["bf16_tflops"], "note": "harness only; not part of a step"}
+            del a, b, c
+
         # ---- timed region: K back-to-back steps; kernel events rotate so every launch is measured
         kev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
         for a, b in kev:
             a.record(stream); b.record(stream)
-        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        sev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]   # step boundaries
         sampler = ClockSampler(local) if rank == 0 else None
         barrier()
         launches0 = B.psa_launch_count()
-        ev0.record(stream)
+        sev[0].record(stream)
         for i in range(args.steps):
             B.psa_profile_events(*kev[i])
             step()
-        ev1.record(stream)
+            sev[i + 1].record(stream)
         barrier()
         launches = B.psa_launch_count() - launches0
         B.psa_profile_events(None, None)
         clocks = sampler.stop() if sampler else None
-        ms_step = ev0.elapsed_time(ev1) / args.steps
+        ms_step = sev[0].elapsed_time(sev[-1]) / args.steps
+        step_ms = [sev[i].elapsed_time(sev[i + 1]) for i in range(args.steps)]
         kernel_ms = float(np.mean([a.elapsed_time(b) for a, b in kev]))
         st, detail = B.psa_last_device_status()
         if st != 0:
@@ -307,6 +362,23 @@ def run_ours(args, w):
             bytes_t = nh * L * HEAD_DIM * 2
             e2e = {"value": world * flops / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
                    "h2d_bytes_per_step": 3 * bytes_t, "d2h_bytes_per_step": bytes_t + nh * L * 4}
+            if rank == 0:
+                # the PCIe floor of such a step: the larger direction's bytes at the measured copy rate
+                # (the two directions overlap on separate copy engines)
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                q.copy_(hq, non_blocking=True)
+                e1.record(stream)
+                torch.cuda.synchronize()
+                h2d_gbs = bytes_t / (e0.elapsed_time(e1) * 1e-3) / 1e9
+                e0.record(stream)
+                hout.copy_(out, non_blocking=True)
+                e1.record(stream)
+                torch.cuda.synchronize()
+                d2h_gbs = bytes_t / (e0.elapsed_time(e1) * 1e-3) / 1e9
+                floor_ms = max(3 * bytes_t / h2d_gbs, (bytes_t + nh * L * 4) / d2h_gbs) / 1e6
+                e2e.update({"h2d_GBps_measured": h2d_gbs, "d2h_GBps_measured": d2h_gbs, "pcie_floor_ms": floor_ms,
+                            "note": "floor = max(h2d bytes / h2d rate, d2h bytes / d2h rate); the kernel hides behind the copies"})
 
     if rank == 0:
         value = world * flops / (ms_max * 1e-3) / 1e12
@@ -317,17 +389,24 @@ def run_ours(args, w):
             for ln in open(tp):
                 if ln.startswith("traffic_bytes_per_launch:"):
                     traffic = int(ln.split(":")[1])
+        issued = issued_flops(nnz, tile)
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": max(args.warmup, 3), "ms_per_step": ms_max, "higher_is_better": True, "scaling": "weak",
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_max, "ms_median": float(np.median(step_ms)),
+            "ms_min": float(np.min(step_ms)), "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": config_of(w, {"l2_policy": "inputs (3.1 GB) exceed L2; no flush needed" if nh * L * 256 * 3 > 2.5e8
-                                    else "inputs fit L2", "peaks": peaks["_source"]}),
+            "config": config_of(w),
+            "computed_flops_per_step": flops, "issued_flops_per_step": issued, "padding_ratio": issued / flops,
             "roofline": {"bound": "tensor", "kernel": "attn_fwd_kernel", "achieved": achieved,
                          "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"],
                          "frac_of_sustained_peak": achieved / peaks["bf16_tflops_sustained"],
+                         "frac_of_datasheet": achieved / DATASHEET_BF16_TFLOPS,
+                         "datasheet_peak": DATASHEET_BF16_TFLOPS,
+                         "datasheet_note": "nominal dense bf16 figure of the part (2.25 PFLOP/s), quoted, not measured",
+                         "issued_tflops": issued / (kernel_ms * 1e-3) / 1e12,
                          "kernel_ms": kernel_ms, "algorithmic_flops_per_launch": flops, "traffic": traffic,
                          "peak_source": peaks["_source"] + " (burst cuBLAS bf16)"},
+            "calibration": calib,
             "clocks": clocks, "gpu_launches": int(launches), "e2e": e2e,
             "context": {"paper_h100_psa_ms": 55.12, "paper_h100_tflops": 29.26 / 55.12e-3,
                         "note": "paper: Table 2, Wan 2.1 14B at 75.00% sparsity on one H100; unpublished per-head parameters"},
@@ -339,9 +418,53 @@ def run_ours(args, w):
                                     "kind": "oracle", "seconds": secs,
                                     "sample": f"{rows} seeded query rows over {heads} heads, each against all {L} keys, "
                                               f"incl. input generation and bf16->fp64 conversion"}
+        if not args.quick and not args.no_configs:
+            del host
+            line["configs"] = time_other_configs(B, WL, torch, dev, peaks, skip=w["name"])
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
+
+
+def time_other_configs(B, WL, torch, dev, peaks, skip):
+    """Kernel-level timing (back-to-back psa_attn_fwd calls, CUDA events) of the other configurations of
+    the benchmark set, with inputs drawn on the device (the time does not depend on the values)."""
+    res = []
+    for name in OTHER_CONFIGS:
+        if name == skip:
+            continue
+        w = WL.workload(name)
+        T, H, W = w["grid"]
+        L, nh, tile = T * H * W, w["n_heads"], w["tile"]
+        params = [tuple(p) for p in w["head_params"]]
+        g = torch.Generator(device=dev).manual_seed(w["seed"])
+        q, k, v = (torch.randn((nh, L, HEAD_DIM), device=dev, generator=g).bfloat16() for _ in range(3))
+        out, lse = torch.empty_like(q), torch.empty((nh, L), dtype=torch.float32, device=dev)
+        flops, dflops = workload_flops(w)
+        iters = 20 if flops < 1e12 else (10 if flops < 6e13 else 4)
+        for _ in range(3):
+            B.psa_attn_fwd(q, k, v, params, w["grid"], tile, SCALE, out=out, lse=lse)
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(iters + 1)]
+        ev[0].record()
+        for i in range(iters):
+            B.psa_attn_fwd(q, k, v, params, w["grid"], tile, SCALE, out=out, lse=lse)
+            ev[i + 1].record()
+        torch.cuda.synchronize()
+        st, detail = B.psa_last_device_status()
+        if st != 0:
+            raise SystemExit(f"{name}: device status {st} {hex(detail)}")
+        ms = [ev[i].elapsed_time(ev[i + 1]) for i in range(iters)]
+        mean = float(np.mean(ms))
+        _, nnz = B.psa_mask_sizes(params, w["grid"], tile)
+        res.append({"workload": name, "grid": w["grid"], "n_heads": nh, "mask_block": tile, "tile_sparsity": w["tile_sparsity"],
+                    "ms": mean, "ms_median": float(np.median(ms)), "ms_min": float(np.min(ms)),
+                    "computed_tflops": flops / (mean * 1e-3) / 1e12,
+                    "frac": flops / (mean * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                    "dense_equiv_tflops": dflops / (mean * 1e-3) / 1e12,
+                    "padding_ratio": issued_flops(nnz, tile) / flops if flops else None})
+        del q, k, v, out, lse
+        torch.cuda.empty_cache()
+    return res
 
 
 def run_report(args):
@@ -517,6 +640,96 @@ def run_search(args, w):
     print(json.dumps(line), flush=True)
 
 
+def run_ulysses(args, w):
+    """The head-sharded call on sequence-sharded inputs (the layout a sequence-parallel DiT keeps its
+    activations in): every rank holds all heads for L / P tokens; one all-to-all per tensor gives each
+    rank heads / P heads with all tokens, the single-GPU kernel runs on them, a second all-to-all
+    returns out and lse.  Total work is fixed ("strong" scaling).  The three phases are timed
+    separately with CUDA events; plain NCCL all-to-all, no peer pointers handed to any kernel."""
+    import torch
+    import torch.distributed as dist
+    from paper_2609_37001_b200 import build
+    build.build()
+    from paper_2609_37001_b200 import binding as B
+    from paper_2609_37001_b200 import replicas as R
+    from paper_2609_37001_b200 import ulysses as U
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=dev)
+    peaks = load_peaks()
+    T, H, W = w["grid"]
+    L, nh, tile = T * H * W, w["n_heads"], w["tile"]
+    if L % world or nh % world:
+        raise SystemExit(f"--ulysses needs tokens ({L}) and heads ({nh}) divisible by the number of ranks ({world})")
+    params = [tuple(p) for p in w["head_params"]]
+    flops, _ = workload_flops(w)
+    g = torch.Generator(device=dev).manual_seed(w["seed"] + rank)
+    q, k, v = (torch.randn((nh, L // world, HEAD_DIM), device=dev, generator=g).bfloat16() for _ in range(3))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def phases():
+        e = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+        e[0].record()
+        qh, kh, vh = (U.seq_to_head_shards(t) for t in (q, k, v))
+        e[1].record()
+        lo, hi = U.local_heads(nh)
+        oh, lh = B.psa_attn_fwd(qh, kh, vh, params[lo:hi], w["grid"], tile, SCALE)
+        e[2].record()
+        o = U.head_to_seq_shards(oh)
+        l = U.head_to_seq_shards(lh.unsqueeze(-1).contiguous()).squeeze(-1)
+        e[3].record()
+        return e, o, l
+
+    for _ in range(max(args.warmup, 3)):
+        phases()
+    barrier()
+    sampler = ClockSampler(local) if rank == 0 else None
+    launches0 = B.psa_launch_count()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    evs = [phases()[0] for _ in range(args.steps)]
+    ev1.record()
+    barrier()
+    launches = B.psa_launch_count() - launches0
+    clocks = sampler.stop() if sampler else None
+    st, detail = B.psa_last_device_status()
+    if st != 0:
+        raise SystemExit(f"device status {st} detail {hex(detail)}")
+    ms = R.max_over_ranks(ev0.elapsed_time(ev1) / args.steps, dev)
+    a2a_in = R.max_over_ranks(float(np.mean([e[0].elapsed_time(e[1]) for e in evs])), dev)
+    attn = R.max_over_ranks(float(np.mean([e[1].elapsed_time(e[2]) for e in evs])), dev)
+    a2a_out = R.max_over_ranks(float(np.mean([e[2].elapsed_time(e[3]) for e in evs])), dev)
+    if rank == 0:
+        per_rank_bytes = nh * (L // world) * HEAD_DIM * 2
+        line = {"metric": METRIC, "value": flops / (ms * 1e-3) / 1e12, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True, "scaling": "strong",
+                "vs_baseline": None, "dtype": "bf16", "data": "synthetic (drawn on the device)",
+                "config": config_of(w, {"parallelism": f"ulysses{world}: sequence-sharded in/out, head-sharded kernel",
+                                         "step": "all_to_all(q,k,v) + psa_attn_fwd + all_to_all(out,lse)"}),
+                "phases_ms": {"all_to_all_in": a2a_in, "attention": attn, "all_to_all_out": a2a_out},
+                "all_to_all_bytes_per_rank": {"in": 3 * per_rank_bytes * (world - 1) // world,
+                                              "out": (per_rank_bytes + nh * (L // world) * 4) * (world - 1) // world},
+                "roofline": {"bound": "tensor", "kernel": "attn_fwd_kernel", "achieved": flops / world / (attn * 1e-3) / 1e12,
+                             "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                             "frac": flops / world / (attn * 1e-3) / 1e12 / peaks["bf16_tflops"], "traffic": None,
+                             "note": "per GPU, attention phase only (planning kernel included)"},
+                "clocks": clocks, "gpu_launches": int(launches), "e2e": None}
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -525,11 +738,19 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="wan14b_720p")
     ap.add_argument("--quick", action="store_true", help="timed region only (no dense/e2e/CPU legs); for profiling")
+    ap.add_argument("--no-configs", action="store_true", help="skip the kernel-level timing of the other configurations")
+    ap.add_argument("--ulysses", action="store_true",
+                    help="time the head-sharded call on sequence-sharded inputs (all-to-all, kernel, all-to-all)")
     ap.add_argument("--report", default=None, metavar="FILE.md",
                     help="time every workload (PSA, dense, mask build) on one GPU and write a markdown table; no JSON line")
     ap.add_argument("--search", type=int, default=0, metavar="N",
                     help="time the PSA-Search inner loop for one head over N seeded candidates instead of the hot path")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "ours" and not args.report and not args.search:
+        # started without a launcher: become one (one process per GPU on this node)
+        from paper_2609_37001_b200 import replicas as R
+        codes = R.launch_ranks([os.path.abspath(__file__)] + sys.argv[1:], args.gpus)
+        raise SystemExit(max(abs(c) for c in codes))
     if args.search:
         from paper_2609_37001_b200 import workloads as WL
         run_search(args, WL.workload(args.workload))
@@ -541,6 +762,8 @@ def main():
     w = WL.workload(args.workload)
     if args.impl == "reference":
         run_reference(args, w)
+    elif args.ulysses:
+        run_ulysses(args, w)
     else:
         run_ours(args, w)
 

@@ -91,7 +91,12 @@ int psa_mask_build(const psa_head_params* params, const psa_problem* prob,
  *   head_params host, n_heads entries
  * Rows whose query block attends no key block get out = 0 and lse = -inf.  Padded
  * positions (Section 3.2, "3D-Padding") are never read from or written to memory.
- * Pointers must be 16-byte aligned.  bf16 inputs, fp32 accumulation. */
+ * Pointers must be 16-byte aligned.  bf16 inputs, fp32 accumulation.
+ * Precondition: the attention kernel takes every SM whole (one CTA with 226 KB of shared memory
+ * and all 512 tensor-memory columns) and its tensor-memory allocation blocks until the columns are
+ * free, so no other kernel that allocates tensor memory may run on the device at the same time
+ * (other processes, or other streams of this process).  Every later wait inside the kernel has
+ * a time limit and is reported through psa_last_device_status(). */
 int psa_attn_fwd(const void* q, const void* k, const void* v, void* out, float* lse,
                  const psa_head_params* head_params, const psa_problem* prob,
                  int T, int H, int W, void* stream);
@@ -118,7 +123,8 @@ int psa_attn_fwd(const void* q, const void* k, const void* v, void* out, float* 
  * array: the planning kernel clears the words that must start at zero and rewrites the rest,
  * so back-to-back calls on one stream are fine, but calls that overlap on the GPU (different
  * streams) race on it.  The status word of this variant is not visible to
- * psa_last_device_status().  No cudaMalloc, cudaFree or other allocating call is made. */
+ * psa_last_device_status(), and the event pair registered with psa_profile_events() is not
+ * recorded by it.  No cudaMalloc, cudaFree or other allocating call is made. */
 int psa_attn_fwd_noalloc(const void* q, const void* k, const void* v, void* out, float* lse,
                          const psa_head_params* head_params, const psa_problem* prob,
                          int T, int H, int W, void* stream, int32_t* status_detail);
@@ -177,7 +183,8 @@ int psa_attn_fwd_joint(const void* q, const void* k, const void* v, void* out, f
  * psa_search_select: the selection -- sort by loss ascending (ties by index), start from the
  * lowest-loss candidate, and among candidates with loss <= alpha move to any strictly sparser one.
  * losses, sparsity: host arrays of n entries (sparsity = excluded fraction of block pairs, e.g. from
- * psa_mask_sizes).  Returns the chosen index (>= 0) or a negative psa_status.  Pure host code.
+ * psa_mask_sizes).  Returns the chosen index (>= 0) or a negative psa_status (PSA_ERR_INVALID_ARG
+ * when a loss is not finite or a sparsity is NaN).  Pure host code.
  *
  * psa_search_select_at_sparsity: the second interface of Section 3.3 -- for a target sparsity, the
  * candidate of minimal loss among those with sparsity >= target (ties by index); PSA_ERR_CAPACITY

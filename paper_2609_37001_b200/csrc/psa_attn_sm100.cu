@@ -21,7 +21,16 @@
 // TMEM (512 columns): S0 | S1 | O0 | O1, 128 fp32 columns each; the bf16 probabilities
 // P_i overwrite the first columns of S_i.  A key slab has 128 keys, or 112/96/64 for the last
 // slab of a block whose token count is not a multiple of 128.
-// Every wait is bounded; on expiry the CTA records a status word and unwinds.
+// Every meeting point inside the kernel's loops is an mbarrier wait with a time limit (2 s of
+// %globaltimer): producer / consumer hand-offs, the merge of a split-KV item, and the gathering
+// of a staged output slab before its TMA store.  On expiry the waiter sets a CTA-wide abort
+// flag; every other waiter sees the flag at its next poll and returns, all roles leave their
+// loops, the load warp waits (bounded) for its TMA loads in flight, the MMA warp waits (bounded)
+// for its MMAs in flight, all threads meet at the one __syncthreads of the teardown, TMEM is
+// freed and the status word reports the timeout.  Not bounded by the kernel: the TMEM allocation
+// at start-up, which blocks while another resident CTA holds tensor memory -- this kernel takes a
+// whole SM (226 KB of shared memory, 512 TMEM columns), so a caller must not run other
+// TMEM-using kernels on the same device concurrently with it.
 // Build-time knob: PSA_EMU_PAIRS (share of exponentials computed by a polynomial on the FMA
 // pipe, default 0).
 #include <cuda.h>
@@ -51,7 +60,8 @@ constexpr int kNumPairBars = kNumSlots;
 constexpr int kBarQFull = 0, kBarQEmpty = 2, kBarPairFull = 4, kBarSlotEmpty = kBarPairFull + kNumPairBars,
               kBarSFull = kBarSlotEmpty + kNumSlots, kBarPHalf = kBarSFull + 2, kBarPReady = kBarPHalf + 2,
               kBarOFull = kBarPReady + 2, kBarOEmpty = kBarOFull + 2, kBarSchedFull = kBarOEmpty + 2,
-              kBarSchedEmpty = kBarSchedFull + 2, kNumBars = (kBarSchedEmpty + 2 + 1) & ~1;
+              kBarSchedEmpty = kBarSchedFull + 2, kBarStage = kBarSchedEmpty + 2, kBarMerge = kBarStage + 2,
+              kBarDrain = kBarMerge + 1, kNumBars = (kBarDrain + 1 + 1) & ~1;
 constexpr uint32_t kOffMeta = kOffBar + kNumBars * 8;           // kMetaRing x 8 words
 constexpr uint32_t kOffMaskT = kOffMeta + kMetaRing * 32;       // kMaxTp / 32 words
 constexpr uint32_t kOffMaskS = kOffMaskT + (kMaxTp / 32) * 4;   // kMaxSp / 32 words
@@ -291,9 +301,6 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
 }
-__device__ __forceinline__ void named_bar_sync(int id, int nthreads) {
-  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
-}
 
 // Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N columns (multiple of 16); A is K-major.
 __host__ __device__ constexpr uint32_t instr_desc(bool b_mn_major, uint32_t n) {
@@ -310,7 +317,7 @@ __device__ __forceinline__ bool elect_one() {
 // Work order: per head, query blocks ranked by attended key-block count (largest first),
 // heads kept together so that concurrently running CTAs share K/V in L2.
 __global__ void __launch_bounds__(256)
-plan_kernel(const HeadParamsArray hp, const Geom g, int head0, int* __restrict__ ws_header,
+plan_kernel(const HeadParamsArray hp, const Geom g, int head0, int clear_status, int* __restrict__ ws_header,
             psa_head_params* __restrict__ hp_dev, WorkItem* __restrict__ items) {
   extern __shared__ int sm[];  // cntT[Tp], cntS[Sp], cnt[NB]
   int* cntT = sm;
@@ -318,7 +325,11 @@ plan_kernel(const HeadParamsArray hp, const Geom g, int head0, int* __restrict__
   int* cnt = cntS + g.Sp;
   const int h = blockIdx.x;
   const psa_head_params p = hp.p[head0 + h];
-  if (h == 0 && threadIdx.x < kWsHeaderWords) ws_header[threadIdx.x] = 0;
+  // The scheduler ticket restarts with every launch; the status words are cleared only by the
+  // first launch of an API call, so that a timeout recorded by an earlier launch of the same call
+  // (a call may need several: more than 128 heads, chunks of a host-tensor call) survives.
+  if (h == 0 && threadIdx.x < kWsHeaderWords && (clear_status || (threadIdx.x != kWsStatus && threadIdx.x != kWsDetail)))
+    ws_header[threadIdx.x] = 0;
   if (threadIdx.x == 0) hp_dev[h] = p;
   for (int a = threadIdx.x; a < g.Tp + g.Sp; a += blockDim.x) {
     int c = 0;
@@ -541,9 +552,12 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
       mbar_init(bar(kBarPReady + i), 128);
       mbar_init(bar(kBarOFull + i), 1);
       mbar_init(bar(kBarOEmpty + i), 128);
+      mbar_init(bar(kBarStage + i), 128);
       mbar_init(bar(kBarSchedFull + i), 1);
       mbar_init(bar(kBarSchedEmpty + i), 9);  // the MMA warp and the eight softmax warps
     }
+    mbar_init(bar(kBarMerge), 128);
+    mbar_init(bar(kBarDrain), 1);
     for (int s = 0; s < kNumPairBars; ++s) mbar_init(bar(kBarPairFull + s), 1);
     for (int s = 0; s < kNumSlots; ++s) mbar_init(bar(kBarSlotEmpty + s), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -1002,6 +1016,16 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
       ++it_o0;
       if (use_o1) ++it_o1;
     }
+    // Every MMA issued so far must have completed before the TMEM allocation is released (after
+    // a timeout some may still be in flight): one more commit, awaited with a bound of its own.
+    if (elect_one()) {
+      tc_commit(bar(kBarDrain));
+      const unsigned long long t0 = globaltimer_ns();
+      while (!mbar_try_wait(bar(kBarDrain), 0u)) {
+        if (globaltimer_ns() - t0 > kTimeoutNs) break;
+      }
+    }
+    __syncwarp();
   }
   } else {
     asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
@@ -1012,6 +1036,8 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
     const uint32_t tS = tmem + lane_addr + (uint32_t)qi * 128u;
     const uint32_t tO = tmem + lane_addr + 256u + (uint32_t)qi * 128u;
     uint32_t it_o0 = 0, it_o1 = 0, cnt_s = 0, kv_g = 0;
+    uint32_t n_stage = 0;   // output slabs staged by this warpgroup so far
+    uint32_t n_merge = 0;   // split-KV merges so far
     bool ok = true;
     const float neg_inf = __int_as_float(0xff800000);
     float2* xchg = reinterpret_cast<float2*>(smem + kOffXchg);
@@ -1064,8 +1090,9 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
       // read both accumulators because they sit in the same TMEM lanes.
       float scale0 = 1.f, scale1 = 0.f;   // weights of O_0 and O_1 in the merged output
       if (split && qi == 1) {
+        // hand (m, l) of the odd key slabs to warpgroup 0 (release / acquire through the barrier)
         xchg[row] = make_float2(m_ref, l);
-        named_bar_sync(3, 256);
+        mbar_arrive(bar(kBarMerge));
         continue;
       }
       ok = mbar_wait_warp(bar(kBarOFull + qi), (qi == 0 ? par_o0 : par_o1), abort_flag, 0x310 + qi);
@@ -1073,7 +1100,9 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
       if (split && use_o1) {
         ok = mbar_wait_warp(bar(kBarOFull + 1), par_o1, abort_flag, 0x312);
         if (!ok) break;
-        named_bar_sync(3, 256);
+        ok = mbar_wait_warp(bar(kBarMerge), n_merge & 1u, abort_flag, 0x313);
+        if (!ok) break;
+        ++n_merge;
         const float2 other = xchg[row];
         const float m_all = fmaxf(m_ref, other.x);
         scale0 = (m_ref == neg_inf) ? 0.f : fast_exp2(m_ref - m_all);
@@ -1142,16 +1171,24 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
           prm.lse[(long long)head * g.Lt + tok] = lse_row;
         }
       }
+      // Every thread's staged row is made visible to the TMA engine; the warpgroup's first warp
+      // waits for all 128 rows (a bounded wait, like every other one) and stores the slab.
       fence_async_smem();
-      named_bar_sync(1 + qi, 128);
-      if ((warp & 3) == 0 && lane == 0) {
-        const uint32_t src = sbase + kOffQ + (uint32_t)qi * kSlabBytes;
-        tma_store_5d(&tms.o[last], src, 0, w0, h0, t0, head);
-        tma_store_5d(&tms.o[last], src + kHalfBytes, 64, w0, h0, t0, head);
-        tma_store_commit();
-        tma_store_wait_read();
-        mbar_arrive(bar(kBarQEmpty + qi));
+      mbar_arrive(bar(kBarStage + qi));
+      if ((warp & 3) == 0) {
+        ok = mbar_wait_warp(bar(kBarStage + qi), n_stage & 1u, abort_flag, 0x320 + qi);
+        if (!ok) break;
+        if (lane == 0) {
+          const uint32_t src = sbase + kOffQ + (uint32_t)qi * kSlabBytes;
+          tma_store_5d(&tms.o[last], src, 0, w0, h0, t0, head);
+          tma_store_5d(&tms.o[last], src + kHalfBytes, 64, w0, h0, t0, head);
+          tma_store_commit();
+          tma_store_wait_read();
+          mbar_arrive(bar(kBarQEmpty + qi));
+        }
+        __syncwarp();
       }
+      ++n_stage;
     }
     if ((warp & 3) == 0 && lane == 0) tma_store_wait_all();
   }
@@ -1194,14 +1231,14 @@ cudaError_t launch_wait_probe(int* ws_header, unsigned long long limit_ns, cudaS
 // ----------------------------------------------------------------------------- launchers
 size_t plan_smem_bytes(const Geom& g) { return sizeof(int) * (size_t)(g.Tp + g.Sp + g.NB); }
 
-cudaError_t launch_plan(const HeadParamsArray& hp, const Geom& g, int head0, int n_heads_here, int* ws_header,
-                        psa_head_params* hp_dev, WorkItem* items, cudaStream_t stream) {
+cudaError_t launch_plan(const HeadParamsArray& hp, const Geom& g, int head0, int n_heads_here, bool clear_status,
+                        int* ws_header, psa_head_params* hp_dev, WorkItem* items, cudaStream_t stream) {
   const size_t smem = plan_smem_bytes(g);
   if (smem > 48 * 1024) {
     cudaError_t e = cudaFuncSetAttribute(plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
   }
-  plan_kernel<<<n_heads_here, 256, smem, stream>>>(hp, g, head0, ws_header, hp_dev, items);
+  plan_kernel<<<n_heads_here, 256, smem, stream>>>(hp, g, head0, clear_status ? 1 : 0, ws_header, hp_dev, items);
   return cudaGetLastError();
 }
 

@@ -3,7 +3,6 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 
-#include <algorithm>
 #include <atomic>
 #include <cmath>
 #include <cstring>
@@ -16,8 +15,8 @@ namespace psa {
 cudaError_t launch_mask_build(const HeadParamsArray& hp, const int* head_bases, const Geom& g, int n_heads_here,
                               uint8_t* block_mask, int* row_ptr, int* col_idx, int total_nnz_through_chunk,
                               int n_sms, cudaStream_t stream, int* launches);
-cudaError_t launch_plan(const HeadParamsArray& hp, const Geom& g, int head0, int n_heads_here, int* ws_header,
-                        psa_head_params* hp_dev, WorkItem* items, cudaStream_t stream);
+cudaError_t launch_plan(const HeadParamsArray& hp, const Geom& g, int head0, int n_heads_here, bool clear_status,
+                        int* ws_header, psa_head_params* hp_dev, WorkItem* items, cudaStream_t stream);
 struct TensorMaps {
   CUtensorMap q[3], k[3], v[3], o[3];  // [0]: full 128-token slab box, [1]: a block's last slab, [2]: text slab
 };
@@ -379,8 +378,9 @@ int psa_mask_build(const psa_head_params* params, const psa_problem* prob, int T
 
 // Planning + attention launches for n_heads heads (in launches of at most kMaxHeads) on the cached
 // per-device workspace.  Arguments are already validated; g_mu is held by the caller.
+// clear_status: this is the first launch sequence of an API call (later ones keep the status word).
 static int run_attn(const void* q, const void* k, const void* v, void* out, float* lse, const psa_head_params* head_params,
-                    int n_heads, const Geom& g, const Layout& lay, cudaStream_t st) {
+                    int n_heads, const Geom& g, const Layout& lay, cudaStream_t st, bool clear_status = true) {
   int dev;
   Workspace* ws;
   int rc = device_info(&dev, &ws);
@@ -410,7 +410,8 @@ static int run_attn(const void* q, const void* k, const void* v, void* out, floa
       return rc;
     Geom gh = g;
     gh.n_heads = n_here;
-    if (launch_plan(hp, gh, 0, n_here, ws_header, hp_dev, items, st) != cudaSuccess) return PSA_ERR_CUDA;
+    if (launch_plan(hp, gh, 0, n_here, clear_status && head0 == 0, ws_header, hp_dev, items, st) != cudaSuccess)
+      return PSA_ERR_CUDA;
     ++g_launches;
     const int n_items = n_here * g.items_per_head;
     if (g_ev_start && g_ev_stop) cudaEventRecord(g_ev_start, st);
@@ -423,8 +424,10 @@ static int run_attn(const void* q, const void* k, const void* v, void* out, floa
   return PSA_OK;
 }
 
-int psa_attn_fwd(const void* q, const void* k, const void* v, void* out, float* lse, const psa_head_params* head_params,
-                 const psa_problem* prob, int T, int H, int W, void* stream) {
+// psa_attn_fwd with the choice of keeping the status word (chunks of one host-tensor call).
+static int attn_fwd_checked(const void* q, const void* k, const void* v, void* out, float* lse,
+                            const psa_head_params* head_params, const psa_problem* prob, int T, int H, int W, void* stream,
+                            bool clear_status) {
   Geom g;
   int rc = make_geom(prob, T, H, W, true, &g);
   if (rc != PSA_OK) return rc;
@@ -438,7 +441,12 @@ int psa_attn_fwd(const void* q, const void* k, const void* v, void* out, float* 
     if (!valid_params(head_params[h])) return PSA_ERR_INVALID_ARG;
   std::lock_guard<std::mutex> lock(g_mu);
   const Layout lay = {prob->stride_head, prob->stride_token, prob->stride_head, prob->stride_token, false};
-  return run_attn(q, k, v, out, lse, head_params, prob->n_heads, g, lay, static_cast<cudaStream_t>(stream));
+  return run_attn(q, k, v, out, lse, head_params, prob->n_heads, g, lay, static_cast<cudaStream_t>(stream), clear_status);
+}
+
+int psa_attn_fwd(const void* q, const void* k, const void* v, void* out, float* lse, const psa_head_params* head_params,
+                 const psa_problem* prob, int T, int H, int W, void* stream) {
+  return attn_fwd_checked(q, k, v, out, lse, head_params, prob, T, H, W, stream, true);
 }
 
 int psa_search_select_at_sparsity(const float* losses, const float* sparsity, int n, float target) {
@@ -483,7 +491,7 @@ int psa_attn_fwd_batched(const void* q, const void* k, const void* v, void* out,
     const long long off = (long long)b * stride_batch;
     rc = run_attn(static_cast<const uint16_t*>(q) + off, static_cast<const uint16_t*>(k) + off,
                   static_cast<const uint16_t*>(v) + off, static_cast<uint16_t*>(out) + off,
-                  lse + (long long)b * nh * g.L, head_params, nh, g, lay, st);
+                  lse + (long long)b * nh * g.L, head_params, nh, g, lay, st, b == 0);
     if (rc != PSA_OK) return rc;
   }
   return PSA_OK;
@@ -555,14 +563,19 @@ int psa_search_losses(const void* q, const void* k, const void* v, const psa_hea
 
 int psa_search_select(const float* losses, const float* sparsity, int n, float alpha) {
   if (!losses || !sparsity || n < 1) return PSA_ERR_INVALID_ARG;
-  // ascending loss, ties by index (stable)
-  std::vector<int> order(n);
-  for (int i = 0; i < n; ++i) order[i] = i;
-  std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return losses[a] < losses[b]; });
-  int best = order[0];
-  for (int i : order)
-    if (losses[i] <= alpha && sparsity[i] > sparsity[best]) best = i;
-  return best;
+  // Algorithm 3 walks the candidates in order of (loss, index), starts at the first and moves to
+  // any strictly sparser one whose loss is within alpha.  Its result, stated directly: if no loss
+  // is within alpha, the candidate of minimal (loss, index); otherwise the sparsest candidate
+  // among those within alpha, ties by minimal (loss, index).
+  int lowest = -1, best = -1;
+  for (int i = 0; i < n; ++i) {
+    if (!std::isfinite(losses[i]) || std::isnan(sparsity[i])) return PSA_ERR_INVALID_ARG;
+    if (lowest < 0 || losses[i] < losses[lowest]) lowest = i;
+    if (losses[i] <= alpha &&
+        (best < 0 || sparsity[i] > sparsity[best] || (sparsity[i] == sparsity[best] && losses[i] < losses[best])))
+      best = i;
+  }
+  return best >= 0 ? best : lowest;
 }
 
 int psa_attn_fwd_noalloc(const void* q, const void* k, const void* v, void* out, float* lse,
@@ -607,7 +620,7 @@ int psa_attn_fwd_noalloc(const void* q, const void* k, const void* v, void* out,
   if ((rc = encode_maps(&tm, q, k, v, out, g, lay, prob->n_heads)) != PSA_OK) return rc;
   // The planning kernel clears the header words (status, ticket) and rewrites the parameter
   // records and every work item of this call, so nothing of the previous call is read.
-  if (launch_plan(hp, g, 0, prob->n_heads, header, hp_dev, items, st) != cudaSuccess) return PSA_ERR_CUDA;
+  if (launch_plan(hp, g, 0, prob->n_heads, true, header, hp_dev, items, st) != cudaSuccess) return PSA_ERR_CUDA;
   ++g_launches;
   if (launch_attn(tm, g, items, hp_dev, header, lse, (int)n_items_ll, ws->n_sms, false, st) != cudaSuccess)
     return PSA_ERR_CUDA;
@@ -678,7 +691,7 @@ int psa_attn_fwd_host(const void* q, const void* k, const void* v, void* out, fl
     if (cudaStreamWaitEvent(st, pipe->ev_in[c], 0) != cudaSuccess) return PSA_ERR_CUDA;
     psa_problem sub = *prob;
     sub.n_heads = nh;
-    const int rc = psa_attn_fwd(dq, dk, dv, dout, d_lse + (size_t)h0 * L, head_params + h0, &sub, T, H, W, stream);
+    const int rc = attn_fwd_checked(dq, dk, dv, dout, d_lse + (size_t)h0 * L, head_params + h0, &sub, T, H, W, stream, c == 0);
     if (rc != PSA_OK) return rc;
     if (cudaEventRecord(pipe->ev_done[c], st) != cudaSuccess) return PSA_ERR_CUDA;
     if (cudaStreamWaitEvent(pipe->d2h, pipe->ev_done[c], 0) != cudaSuccess) return PSA_ERR_CUDA;

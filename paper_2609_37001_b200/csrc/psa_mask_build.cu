@@ -1,6 +1,8 @@
 // psa_mask_build: block mask and GetKVBlocks index lists from the stripe parameters
 // (Algorithm 1 evaluated on block coordinates; Algorithm 2, producer side).
-// Integer work only, bound by the HBM writes of the mask bytes and the column ids.
+// Integer work only.  Two kernels: a register-only one for block grids of at most 32 x 32
+// coordinates per axis pair (mask_build_small_kernel, further down), and the general one
+// described here.
 //
 // The two conditions of Algorithm 1 depend only on coordinate differences, so each block of
 // threads first tabulates, for its head, "does difference d attend" for every temporal and
@@ -128,11 +130,95 @@ mask_build_kernel(const HeadParamsArray hp, const HeadBases hb, const Geom g, in
     row_ptr[(long long)n_heads_here * g.NB] = total_nnz;
 }
 
+// Fast path for block grids with at most 32 temporal and 32 spatial block coordinates (all the
+// paper's shapes): no shared memory and no block-wide barrier.  Every warp rebuilds the head's
+// two difference bitsets with four ballots (bit d + n - 1 of an axis' set = "difference d
+// attends"), so the key coordinates a query coordinate x attends are one shift away:
+// (set >> (n - 1 - x)) & ((1 << n) - 1).  Row counts are popcounts, their prefix sums one warp
+// scan.  A warp then owns whole rows: the byte mask is written 32 key blocks per step, and the
+// column list as the sorted Cartesian product -- for every attended temporal coordinate (a
+// warp-uniform loop over set bits) the lanes whose spatial bit is set store tk * S' + lane at
+// their rank, i.e. consecutive addresses.
+__global__ void __launch_bounds__(256)
+mask_build_small_kernel(const HeadParamsArray hp, const HeadBases hb, const Geom g, int n_heads_here, int rows_per_warp,
+                        uint8_t* __restrict__ block_mask, int* __restrict__ row_ptr, int* __restrict__ col_idx,
+                        int total_nnz) {
+  const int h = blockIdx.y;
+  const psa_head_params p = hp.p[h];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+  const int Tp = g.Tp, Sp = g.Sp;
+  const unsigned long long setT =
+      (unsigned long long)__ballot_sync(0xffffffffu, lane < 2 * Tp - 1 && axis_attends(lane - (Tp - 1), p.Tw, p.To, p.Ts)) |
+      ((unsigned long long)__ballot_sync(0xffffffffu, lane + 32 < 2 * Tp - 1 && axis_attends(lane + 32 - (Tp - 1), p.Tw, p.To, p.Ts)) << 32);
+  const unsigned long long setS =
+      (unsigned long long)__ballot_sync(0xffffffffu, lane < 2 * Sp - 1 && axis_attends(lane - (Sp - 1), p.Sw, p.So, p.Ss)) |
+      ((unsigned long long)__ballot_sync(0xffffffffu, lane + 32 < 2 * Sp - 1 && axis_attends(lane + 32 - (Sp - 1), p.Sw, p.So, p.Ss)) << 32);
+  const unsigned maskT = Tp == 32 ? 0xffffffffu : ((1u << Tp) - 1u), maskS = Sp == 32 ? 0xffffffffu : ((1u << Sp) - 1u);
+  auto rowT = [&](int x) -> unsigned { return (unsigned)(setT >> (Tp - 1 - x)) & maskT; };
+  auto rowS = [&](int x) -> unsigned { return (unsigned)(setS >> (Sp - 1 - x)) & maskS; };
+  // lane x holds the count of coordinate x and the exclusive prefix of the counts before it
+  const int cntT = lane < Tp ? __popc(rowT(lane)) : 0, cntS = lane < Sp ? __popc(rowS(lane)) : 0;
+  int incT = cntT, incS = cntS;
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const int a = __shfl_up_sync(0xffffffffu, incT, off), b = __shfl_up_sync(0xffffffffu, incS, off);
+    if (lane >= off) { incT += a; incS += b; }
+  }
+  const int preT = incT - cntT, preS = incS - cntS;
+  const int sumS = __shfl_sync(0xffffffffu, incS, 31);
+  const int q0 = (blockIdx.x * nwarps + warp) * rows_per_warp;
+  const int q1 = min(g.NB, q0 + rows_per_warp);
+  const long long nb2 = (long long)g.NB * g.NB;
+  const unsigned lane_lt = (1u << lane) - 1u;
+  for (int qb = q0; qb < q1; ++qb) {
+    const int tq = qb / Sp, sq = qb - tq * Sp;
+    const unsigned mT = rowT(tq), mS = rowS(sq);
+    const int cT = __shfl_sync(0xffffffffu, cntT, tq), pT = __shfl_sync(0xffffffffu, preT, tq);
+    const int cS = __shfl_sync(0xffffffffu, cntS, sq), pS = __shfl_sync(0xffffffffu, preS, sq);
+    int pos = hb.base[h] + pT * sumS + cT * pS;
+    if (row_ptr && lane == 0) row_ptr[(long long)h * g.NB + qb] = pos;
+    if (block_mask) {
+      uint8_t* mrow = block_mask + (long long)h * nb2 + (long long)qb * g.NB;
+      int tk = lane / Sp, sk = lane - tk * Sp;       // coordinates of key block `lane`
+      const int dt = 32 / Sp, ds = 32 - dt * Sp;    // advance of 32 key blocks
+      for (int kb = lane; kb < g.NB; kb += 32) {
+        mrow[kb] = (uint8_t)(((mT >> tk) & (mS >> sk)) & 1u);
+        tk += dt;
+        sk += ds;
+        if (sk >= Sp) { sk -= Sp; ++tk; }
+      }
+    }
+    if (col_idx) {
+      const bool mine = (mS >> lane) & 1u;
+      const int rank = __popc(mS & lane_lt);
+      for (unsigned rest = mT; rest; rest &= rest - 1u) {
+        const int tk = __ffs(rest) - 1;
+        if (mine) col_idx[pos + rank] = tk * Sp + lane;
+        pos += cS;
+      }
+    }
+  }
+  if (row_ptr && blockIdx.x == 0 && h == n_heads_here - 1 && threadIdx.x == 0)
+    row_ptr[(long long)n_heads_here * g.NB] = total_nnz;
+}
+
 cudaError_t launch_mask_build(const HeadParamsArray& hp, const int* head_bases, const Geom& g, int n_heads_here,
                               uint8_t* block_mask, int* row_ptr, int* col_idx, int total_nnz_through_chunk,
                               int n_sms, cudaStream_t stream, int* launches) {
   HeadBases hb;
   for (int h = 0; h < kMaxHeads; ++h) hb.base[h] = h < n_heads_here ? head_bases[h] : 0;
+  if (g.Tp <= 32 && g.Sp <= 32) {
+    // a few rows per warp: enough warps to fill the machine, little per-warp set-up to repeat
+    const int warps_wanted = 8 * 4 * n_sms;   // 8 warps per block, 4 blocks per SM
+    int rows_per_warp = (int)(((long long)g.NB * n_heads_here + warps_wanted - 1) / warps_wanted);
+    if (rows_per_warp < 1) rows_per_warp = 1;
+    const int rows_per_block = 8 * rows_per_warp;
+    dim3 grid((g.NB + rows_per_block - 1) / rows_per_block, n_heads_here);
+    mask_build_small_kernel<<<grid, 256, 0, stream>>>(hp, hb, g, n_heads_here, rows_per_warp, block_mask, row_ptr, col_idx,
+                                                      total_nnz_through_chunk);
+    ++*launches;
+    return cudaGetLastError();
+  }
   const size_t smem = tables_bytes(g);
   if (smem > 48 * 1024) {
     cudaError_t e = cudaFuncSetAttribute(mask_build_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);

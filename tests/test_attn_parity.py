@@ -2,6 +2,10 @@
 
 Tolerances (bf16 inputs, fp32 accumulation, bf16 probabilities): out max-abs <= 2e-2,
 mean-abs <= 2e-3, lse max-abs <= 1e-3, plus a relative L2 bound of 1e-2 on the output.
+The output is rounded to bf16 (relative precision 2^-9), so where an output element exceeds 1 in
+magnitude -- only the sharply peaked test inputs produce such rows -- its error is measured
+relative to that magnitude; with i.i.d. N(0,1) inputs every |out| is below 1 and the absolute
+tolerances apply unchanged.
 Small workloads are compared on every row; the full-size workloads on seeded sampled rows
 (whole query slabs at grid corners plus random rows), each against all keys."""
 import math
@@ -51,7 +55,7 @@ def _compare(out_rows, lse_rows, ref_out, ref_lse, what):
     empty = np.isneginf(ref_lse)
     assert np.array_equal(np.isneginf(lse_rows), empty), what
     assert np.all(out_rows[empty] == 0), what
-    err = np.abs(out_rows - ref_out)
+    err = np.abs(out_rows - ref_out) / np.maximum(1.0, np.abs(ref_out))
     assert err.max() <= OUT_MAX, (what, err.max())
     assert err.mean() <= OUT_MEAN, (what, err.mean())
     ok = ~empty
@@ -112,6 +116,14 @@ def test_small_shapes_every_row(B, grid, tile, params):
 def test_peaked_inputs_every_row(B):
     """q, k scaled so the softmax is concentrated: a wrongly skipped or included tile moves the output by O(1)."""
     _run_and_check(B, [(2, 0, 3, 2, 0, 3), (1, -1, INF, 3, 0, INF)], (8, 16, 32), (1, 16, 16), seed=0x78, gain=2.0)
+
+
+@pytest.mark.parametrize("grid,tile", [((4, 45, 32), (1, 15, 16)), ((6, 16, 32), (3, 8, 16))])
+def test_sharply_peaked_inputs_every_row(B, grid, tile):
+    """q and k scaled by 4: the softmax of a row is dominated by a handful of keys, so a missing or
+    extra tile, or a rescale applied to the wrong accumulator, shows as an O(1) error.  Blocks of
+    128 + 112 tokens and of three 128-token slabs (two-slab and single-slab work items)."""
+    _run_and_check(B, [(2, 0, 3, 2, 0, 3), (1, -1, INF, 3, 0, INF), (2, 1, INF, 1, 0, 2)], grid, tile, seed=0x7C, gain=4.0)
 
 
 def test_strided_token_major_layout(B):

@@ -37,6 +37,9 @@ def _expected_counts(params, grid, tile):
     ((5, 13, 19), (1, 16, 16), [(2, 0, INF, 2, 0, INF), (1, 1, 2, 1, -1, 3), (1, 2, INF, 1, 0, INF)]),
     ((6, 20, 40), (3, 8, 16), [(1, 0, 2, 2, 1, 3), (2, -1, INF, 1, 0, 5)]),
     ((21, 45, 79), (1, 16, 16), [(9, 0, INF, 2, 0, 6), (1, -2, 2, 1, 0, 5)]),
+    # the headline block at both 720p shapes: 128 + 112-token slabs on an unpadded 45-row grid
+    ((21, 45, 80), (1, 15, 16), [(5, 0, INF, 2, 0, 6), (2, 1, 3, 1, -1, 5)]),
+    ((33, 45, 80), (1, 15, 16), [(7, -1, INF, 3, 0, 6), (1, 0, 2, 2, 1, INF)]),
 ])
 def test_zero_query_counts_and_block_code_values(B, grid, tile, params):
     T, H, W = grid

@@ -57,3 +57,34 @@ def test_single_process_identity_and_uneven_shards():
     assert cuts[0][0] == 0 and cuts[-1][1] == 24
     assert all(a[1] == b[0] for a, b in zip(cuts, cuts[1:]))
     assert sorted(hi - lo for lo, hi in cuts) == [4, 5, 5, 5, 5]
+
+
+_RANK_SCRIPT = r"""
+import os, sys
+import torch, torch.distributed as dist
+dist.init_process_group("gloo")          # env:// rendezvous: everything comes from the launcher's environment
+t = torch.tensor([float(dist.get_rank() + 1)])
+dist.all_reduce(t)
+ok = (t.item() == sum(range(1, dist.get_world_size() + 1)) and os.environ["LOCAL_RANK"] == os.environ["RANK"]
+      and os.environ["MASTER_ADDR"] == "127.0.0.1")
+if dist.get_rank() == 0:
+    print("RESULT", dist.get_world_size(), int(ok), flush=True)
+dist.destroy_process_group()
+sys.exit(0 if ok else 3)
+"""
+
+
+def test_launcher_builds_rank_environments_and_starts_the_ranks(tmp_path, capfd):
+    """bench.py --gpus N without a launcher starts its own ranks through replicas.launch_ranks: every rank
+    must find a complete env:// rendezvous (checked with two gloo ranks), and a failing rank must surface."""
+    env = R.rank_env(1, 4, 29555, base={"PATH": "/bin"})
+    assert env["RANK"] == "1" and env["LOCAL_RANK"] == "1" and env["WORLD_SIZE"] == "4"
+    assert env["MASTER_ADDR"] == "127.0.0.1" and env["MASTER_PORT"] == "29555" and env["PATH"] == "/bin"
+    script = tmp_path / "rank.py"
+    script.write_text(_RANK_SCRIPT)
+    codes = R.launch_ranks([str(script)], 2, timeout=300)
+    assert codes == [0, 0]
+    assert "RESULT 2 1" in capfd.readouterr().out          # rank 0's stdout is inherited, the others' is dropped
+    bad = tmp_path / "bad.py"
+    bad.write_text("import os, sys\nsys.exit(5 if os.environ['RANK'] == '1' else 0)\n")
+    assert R.launch_ranks([str(bad)], 2, timeout=60) == [0, 5]

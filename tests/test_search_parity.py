@@ -133,6 +133,10 @@ def test_select_matches_oracle_and_hand_examples(B):
         assert B.psa_search_select_at_sparsity(ls, sp, target) == O.search_select_at_sparsity(ls, sp, target)
     with pytest.raises(ValueError):
         B.psa_search_select([0.1], [0.1, 0.2], 0.5)
+    # a loss that is not finite has no place in the order: rejected, not sorted
+    for bad in (float("nan"), float("inf")):
+        with pytest.raises(RuntimeError):
+            B.psa_search_select([0.25, bad, 0.125], [0.5, 0.75, 0.25], 0.5)
 
 
 @pytest.mark.gpu
@@ -148,9 +152,22 @@ def test_losses_at_full_size_agree_with_the_attention_entry_point(B):
     cands = [tuple(w["head_params"][h]) for h in (0, 2, 12)]
     bits = {n: WL.head_bits(w["seed"], n, 3, L) for n in ("q", "k", "v")}
     q, k, v = (_to_dev(bits[n]) for n in ("q", "k", "v"))
-    got = B.psa_search_losses(q, k, v, cands, grid, tile, SCALE).cpu().numpy().astype(np.float64)
+    scratch = torch.empty(B.psa_search_scratch_bytes(len(cands), grid), dtype=torch.uint8, device="cuda")
+    got = B.psa_search_losses(q, k, v, cands, grid, tile, SCALE, scratch=scratch).cpu().numpy().astype(np.float64)
     assert B.psa_last_device_status()[0] == 0
     Tp, Hp, Wp = O.block_grid(T, H, W, tuple(tile))
+    # The candidate outputs (and full attention's) that the losses were reduced from sit at the start
+    # of the scratch buffer, [n_cand + 1][L][128] bf16: sampled rows of each against the fp64 oracle.
+    n_out = (len(cands) + 1) * L * 128
+    outs = scratch[:2 * n_out].view(torch.bfloat16).view(len(cands) + 1, L, 128)
+    qf, kf, vf = (O.bf16_bits_to_f64(bits[n]) for n in ("q", "k", "v"))
+    rows = WL.sample_rows(w["seed"], 3, L, 24)
+    for c, p in enumerate(list(cands) + [(Tp, 0, INF, Hp * Wp, 0, INF)]):
+        ro, _ = O.attention_rows(qf, kf, vf, rows, tuple(p), T, H, W, tuple(tile), SCALE)
+        mine = outs[c][torch.tensor(rows, device="cuda")].float().cpu().numpy().astype(np.float64)
+        err = np.abs(mine - ro)
+        assert err.max() <= 2e-2 and err.mean() <= 2e-3, (c, err.max(), err.mean())
+        assert np.linalg.norm(mine - ro) <= 1e-2 * np.linalg.norm(ro), c
     full, _ = B.psa_attn_fwd(q[None], k[None], v[None], [(Tp, 0, INF, Hp * Wp, 0, INF)], grid, tile, SCALE)
     for c, p in enumerate(cands):
         o, _ = B.psa_attn_fwd(q[None], k[None], v[None], [p], grid, tile, SCALE)
