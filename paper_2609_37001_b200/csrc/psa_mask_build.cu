@@ -131,28 +131,32 @@ mask_build_kernel(const HeadParamsArray hp, const HeadBases hb, const Geom g, in
 }
 
 // Fast path for block grids with at most 32 temporal and 32 spatial block coordinates (all the
-// paper's shapes): no shared memory and no block-wide barrier.  Every warp rebuilds the head's
-// two difference bitsets with four ballots (bit d + n - 1 of an axis' set = "difference d
-// attends"), so the key coordinates a query coordinate x attends are one shift away:
+// paper's shapes): no shared-memory tables and no block-wide barrier.  The host evaluates the
+// two axis conditions of Algorithm 1 once per head for every coordinate difference and hands
+// the kernel two 64-bit sets per head (bit d + n - 1 of an axis' set = "difference d attends"),
+// so the key coordinates a query coordinate x attends are one shift away:
 // (set >> (n - 1 - x)) & ((1 << n) - 1).  Row counts are popcounts, their prefix sums one warp
 // scan.  A warp then owns whole rows: the byte mask is written 32 key blocks per step, and the
-// column list as the sorted Cartesian product -- for every attended temporal coordinate (a
-// warp-uniform loop over set bits) the lanes whose spatial bit is set store tk * S' + lane at
-// their rank, i.e. consecutive addresses.
+// column list -- the sorted Cartesian product of the two attended coordinate sets -- 32
+// consecutive entries per step.
+struct HeadSets {
+  unsigned long long setT[kMaxHeads], setS[kMaxHeads];
+  int base[kMaxHeads];  // number of attended block pairs of all earlier heads
+};
+
 __global__ void __launch_bounds__(256)
-mask_build_small_kernel(const HeadParamsArray hp, const HeadBases hb, const Geom g, int n_heads_here, int rows_per_warp,
+mask_build_small_kernel(const HeadSets hs, const Geom g, int n_heads_here, int rows_per_warp,
                         uint8_t* __restrict__ block_mask, int* __restrict__ row_ptr, int* __restrict__ col_idx,
                         int total_nnz) {
   const int h = blockIdx.y;
-  const psa_head_params p = hp.p[h];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
   const int Tp = g.Tp, Sp = g.Sp;
-  const unsigned long long setT =
-      (unsigned long long)__ballot_sync(0xffffffffu, lane < 2 * Tp - 1 && axis_attends(lane - (Tp - 1), p.Tw, p.To, p.Ts)) |
-      ((unsigned long long)__ballot_sync(0xffffffffu, lane + 32 < 2 * Tp - 1 && axis_attends(lane + 32 - (Tp - 1), p.Tw, p.To, p.Ts)) << 32);
-  const unsigned long long setS =
-      (unsigned long long)__ballot_sync(0xffffffffu, lane < 2 * Sp - 1 && axis_attends(lane - (Sp - 1), p.Sw, p.So, p.Ss)) |
-      ((unsigned long long)__ballot_sync(0xffffffffu, lane + 32 < 2 * Sp - 1 && axis_attends(lane + 32 - (Sp - 1), p.Sw, p.So, p.Ss)) << 32);
+  if (row_ptr && blockIdx.x == 0 && h == n_heads_here - 1 && threadIdx.x == 0)
+    row_ptr[(long long)n_heads_here * g.NB] = total_nnz;
+  const int q0 = (blockIdx.x * nwarps + warp) * rows_per_warp;
+  const int q1 = min(g.NB, q0 + rows_per_warp);
+  if (q0 >= q1) return;
+  const unsigned long long setT = hs.setT[h], setS = hs.setS[h];
   const unsigned maskT = Tp == 32 ? 0xffffffffu : ((1u << Tp) - 1u), maskS = Sp == 32 ? 0xffffffffu : ((1u << Sp) - 1u);
   auto rowT = [&](int x) -> unsigned { return (unsigned)(setT >> (Tp - 1 - x)) & maskT; };
   auto rowS = [&](int x) -> unsigned { return (unsigned)(setS >> (Sp - 1 - x)) & maskS; };
@@ -166,40 +170,55 @@ mask_build_small_kernel(const HeadParamsArray hp, const HeadBases hb, const Geom
   }
   const int preT = incT - cntT, preS = incS - cntS;
   const int sumS = __shfl_sync(0xffffffffu, incS, 31);
-  const int q0 = (blockIdx.x * nwarps + warp) * rows_per_warp;
-  const int q1 = min(g.NB, q0 + rows_per_warp);
-  const long long nb2 = (long long)g.NB * g.NB;
+  __shared__ int strips[8 * 64];           // per warp: the r-th attended temporal / spatial coordinate
+  int* strip = strips + warp * 64;
+  int tq_tab = -1;                         // query coordinate the temporal table was built for
   const unsigned lane_lt = (1u << lane) - 1u;
+  // coordinates of key block `lane`, and the advance of 32 key blocks
+  const int tk0 = lane / Sp, sk0 = lane - tk0 * Sp;
+  const int dt = 32 / Sp, ds = 32 - dt * Sp;
+  int tq = q0 / Sp, sq = q0 - tq * Sp;
+  uint8_t* mrow = block_mask ? block_mask + ((long long)h * g.NB + q0) * g.NB : nullptr;
+  int* rp = row_ptr ? row_ptr + (long long)h * g.NB + q0 : nullptr;
   for (int qb = q0; qb < q1; ++qb) {
-    const int tq = qb / Sp, sq = qb - tq * Sp;
     const unsigned mT = rowT(tq), mS = rowS(sq);
     const int cT = __shfl_sync(0xffffffffu, cntT, tq), pT = __shfl_sync(0xffffffffu, preT, tq);
     const int cS = __shfl_sync(0xffffffffu, cntS, sq), pS = __shfl_sync(0xffffffffu, preS, sq);
-    int pos = hb.base[h] + pT * sumS + cT * pS;
-    if (row_ptr && lane == 0) row_ptr[(long long)h * g.NB + qb] = pos;
-    if (block_mask) {
-      uint8_t* mrow = block_mask + (long long)h * nb2 + (long long)qb * g.NB;
-      int tk = lane / Sp, sk = lane - tk * Sp;       // coordinates of key block `lane`
-      const int dt = 32 / Sp, ds = 32 - dt * Sp;    // advance of 32 key blocks
+    const int pos = hs.base[h] + pT * sumS + cT * pS;
+    if (rp && lane == 0) *rp = pos;
+    if (mrow) {
+      int tk = tk0, sk = sk0;
       for (int kb = lane; kb < g.NB; kb += 32) {
         mrow[kb] = (uint8_t)(((mT >> tk) & (mS >> sk)) & 1u);
         tk += dt;
         sk += ds;
         if (sk >= Sp) { sk -= Sp; ++tk; }
       }
+      mrow += g.NB;
     }
-    if (col_idx) {
-      const bool mine = (mS >> lane) & 1u;
-      const int rank = __popc(mS & lane_lt);
-      for (unsigned rest = mT; rest; rest &= rest - 1u) {
-        const int tk = __ffs(rest) - 1;
-        if (mine) col_idx[pos + rank] = tk * Sp + lane;
-        pos += cS;
+    if (col_idx && cT * cS > 0) {
+      // Entry e of the row's list is (the (e / cS)-th attended temporal coordinate, the
+      // (e % cS)-th attended spatial one).  "The r-th set bit" comes from two 32-entry tables in the
+      // warp's strip (a lane whose bit is set writes its index at its rank; the temporal table
+      // only changes with tq); e / cS is a multiply and a shift (e < 1024, cS <= 32).  The list is
+      // then written 32 consecutive entries per store.
+      if (tq != tq_tab) {
+        if ((mT >> lane) & 1u) strip[__popc(mT & lane_lt)] = lane;
+        tq_tab = tq;
       }
+      if ((mS >> lane) & 1u) strip[32 + __popc(mS & lane_lt)] = lane;
+      __syncwarp();
+      const int count = cT * cS;
+      const unsigned inv = (65536u + (unsigned)cS - 1u) / (unsigned)cS;
+      for (int e = lane; e < count; e += 32) {
+        const int it = (int)(((unsigned)e * inv) >> 16), is = e - it * cS;
+        col_idx[pos + e] = strip[it] * Sp + strip[32 + is];
+      }
+      __syncwarp();
     }
+    if (rp) ++rp;
+    if (++sq == Sp) { sq = 0; ++tq; }
   }
-  if (row_ptr && blockIdx.x == 0 && h == n_heads_here - 1 && threadIdx.x == 0)
-    row_ptr[(long long)n_heads_here * g.NB] = total_nnz;
 }
 
 cudaError_t launch_mask_build(const HeadParamsArray& hp, const int* head_bases, const Geom& g, int n_heads_here,
@@ -208,14 +227,28 @@ cudaError_t launch_mask_build(const HeadParamsArray& hp, const int* head_bases, 
   HeadBases hb;
   for (int h = 0; h < kMaxHeads; ++h) hb.base[h] = h < n_heads_here ? head_bases[h] : 0;
   if (g.Tp <= 32 && g.Sp <= 32) {
-    // a few rows per warp: enough warps to fill the machine, little per-warp set-up to repeat
-    const int warps_wanted = 8 * 4 * n_sms;   // 8 warps per block, 4 blocks per SM
+    HeadSets hs;
+    for (int h = 0; h < kMaxHeads; ++h) {
+      unsigned long long st = 0, ss = 0;
+      if (h < n_heads_here) {
+        const psa_head_params& p = hp.p[h];
+        for (int i = 0; i < 2 * g.Tp - 1; ++i)
+          if (axis_attends(i - (g.Tp - 1), p.Tw, p.To, p.Ts)) st |= 1ull << i;
+        for (int i = 0; i < 2 * g.Sp - 1; ++i)
+          if (axis_attends(i - (g.Sp - 1), p.Sw, p.So, p.Ss)) ss |= 1ull << i;
+      }
+      hs.setT[h] = st;
+      hs.setS[h] = ss;
+      hs.base[h] = h < n_heads_here ? head_bases[h] : 0;
+    }
+    // one to three rows per warp: the per-row work is a dependent chain, so more warps beat longer ones
+    const int warps_wanted = 8 * 8 * n_sms;
     int rows_per_warp = (int)(((long long)g.NB * n_heads_here + warps_wanted - 1) / warps_wanted);
     if (rows_per_warp < 1) rows_per_warp = 1;
     const int rows_per_block = 8 * rows_per_warp;
     dim3 grid((g.NB + rows_per_block - 1) / rows_per_block, n_heads_here);
-    mask_build_small_kernel<<<grid, 256, 0, stream>>>(hp, hb, g, n_heads_here, rows_per_warp, block_mask, row_ptr, col_idx,
-                                                      total_nnz_through_chunk);
+    mask_build_small_kernel<<<grid, 256, 0, stream>>>(
+        hs, g, n_heads_here, rows_per_warp, block_mask, row_ptr, col_idx, total_nnz_through_chunk);
     ++*launches;
     return cudaGetLastError();
   }
