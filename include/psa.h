@@ -133,9 +133,10 @@ int psa_attn_fwd_noalloc(const void* q, const void* k, const void* v, void* out,
  * copies to overlap) into the caller's device staging buffers d_q, d_k, d_v, runs
  * psa_attn_fwd into d_out / d_lse and copies the results to out / lse (host), ordered
  * after the work already on `stream`, then synchronises `stream`.  When heads are the
- * outermost dimension of the layout the call is pipelined over up to 8 chunks of heads on
- * two internal helper streams: the next chunk is copied in and the previous one copied out
- * while a chunk computes.
+ * outermost dimension of the layout the call is pipelined over chunks of heads (20 by default,
+ * from a measured sweep; the environment variable PSA_HOST_CHUNKS overrides it) on two internal
+ * helper streams: the next chunk is copied in and the previous one copied out while a chunk
+ * computes.
  * Each staging buffer must hold the full strided extent of its tensor:
  * (n_heads-1)*stride_head + (L-1)*stride_token + head_dim elements. */
 int psa_attn_fwd_host(const void* q, const void* k, const void* v, void* out, float* lse,
