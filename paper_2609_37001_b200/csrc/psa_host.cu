@@ -692,9 +692,15 @@ int psa_attn_fwd_host(const void* q, const void* k, const void* v, void* out, fl
   if (cudaEventRecord(pipe->ev_start, st) != cudaSuccess) return PSA_ERR_CUDA;
   if (cudaStreamWaitEvent(pipe->h2d, pipe->ev_start, 0) != cudaSuccess) return PSA_ERR_CUDA;
   if (cudaStreamWaitEvent(pipe->d2h, pipe->ev_start, 0) != cudaSuccess) return PSA_ERR_CUDA;
+  // The first and the last chunks are the exposed ones, so the call starts and ends with
+  // single-head chunks (two at each end, when the regular chunk is larger than that).
+  const int n_edge = (per >= 2 && prob->n_heads >= 4 * per) ? 2 : 0;
   int c = 0;
-  for (int h0 = 0; h0 < prob->n_heads; h0 += per, ++c) {
-    const int nh = prob->n_heads - h0 < per ? prob->n_heads - h0 : per;
+  for (int h0 = 0, nh = 0; h0 < prob->n_heads; h0 += nh, ++c) {
+    const int left = prob->n_heads - h0;
+    if (h0 < n_edge || left <= n_edge) nh = 1;
+    else nh = left - n_edge < per ? left - n_edge : per;
+    if (c >= kHostChunks) return PSA_ERR_UNSUPPORTED;
     const size_t off = (size_t)h0 * prob->stride_head;                       // elements
     const size_t bytes = ((size_t)(nh - 1) * prob->stride_head + head_span) * 2;
     const uint16_t *hq = static_cast<const uint16_t*>(q) + off, *hk = static_cast<const uint16_t*>(k) + off,

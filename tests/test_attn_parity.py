@@ -163,6 +163,7 @@ def _sampled_rows(grid, tile, seed):
 
 @pytest.mark.parametrize("name,heads", [
     ("wan13b_480p", None),
+    ("wan13b_480p_b3x32x4", [0, 4, 7, 11]),
     ("wan14b_720p", list(range(0, 40, 5))),
     ("wan14b_720p_b1x16x16", [2, 17, 31]),
     ("wan14b_720p_b3x8x16", [0, 13, 26]),
