@@ -43,7 +43,8 @@ typedef enum {
   PSA_ERR_UNSUPPORTED = -2, /* head_dim != 128, unsupported tile shape, not sm_100             */
   PSA_ERR_CAPACITY = -3,    /* col_capacity < nnz                                             */
   PSA_ERR_CUDA = -4,        /* a CUDA runtime/driver call failed                              */
-  PSA_ERR_TIMEOUT = -5      /* a bounded device-side wait expired (see psa_last_device_status) */
+  PSA_ERR_TIMEOUT = -5,     /* a bounded device-side wait expired (see psa_last_device_status) */
+  PSA_ERR_INTERNAL = -6     /* checked build only: a kernel-side index / coordinate check failed    */
 } psa_status;
 
 /* Six stripe parameters of one head, in block units (Section 3.2).  Ts == 0 / Ss == 0

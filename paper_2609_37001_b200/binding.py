@@ -21,6 +21,7 @@ PSA_ERR_UNSUPPORTED = -2
 PSA_ERR_CAPACITY = -3
 PSA_ERR_CUDA = -4
 PSA_ERR_TIMEOUT = -5
+PSA_ERR_INTERNAL = -6
 
 
 class PsaError(RuntimeError):

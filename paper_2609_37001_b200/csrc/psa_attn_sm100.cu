@@ -313,6 +313,20 @@ __device__ __forceinline__ bool elect_one() {
   return pred != 0;
 }
 
+// Checked build (-DPSA_DEBUG_CHECKS; the stand-in for a memory checker): every global store index,
+// TMA coordinate, ring / table index and TMEM column range computed by the kernel is verified before
+// use.  A violation records PSA_ERR_INTERNAL with a code naming the site in the status word and the
+// access is skipped -- nothing traps.  In the regular build the checks compile to `true`.
+#ifdef PSA_DEBUG_CHECKS
+__device__ __noinline__ bool dbg_fail(int* ws_header, int code) {
+  if (atomicCAS(ws_header + kWsStatus, 0, (int)PSA_ERR_INTERNAL) == 0) ws_header[kWsDetail] = code;
+  return false;
+}
+#define PSA_CHECKED(cond, code) ((cond) ? true : dbg_fail(prm.ws_header, (code)))
+#else
+#define PSA_CHECKED(cond, code) true
+#endif
+
 // ----------------------------------------------------------------------------- planning
 // Work order: per head, query blocks ranked by attended key-block count (largest first),
 // heads kept together so that concurrently running CTAs share K/V in L2.
@@ -623,6 +637,12 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
       wi.w = __shfl_sync(0xffffffffu, wi.w, 0);
       if (wi.x < 0) break;
       const int head = wi.x, qb = wi.y, sub0 = wi.w & 0xffff, nq = (wi.w >> 16) & 0xff;
+      if (!PSA_CHECKED(head < g.n_heads && qb >= 0 && qb <= g.NB && nq >= 1 && nq <= 2 &&
+                       sub0 + nq <= ((wi.w >> 25) & 1 ? g.n_ts : g.n_sub), 0xD04)) {
+        if (lane == 0) atomicCAS((int*)abort_flag, 0, 0xD04);   // a malformed item: stop this CTA through the abort path
+        ok = false;
+        break;
+      }
       const int lag = ((wi.w >> 24) & 1) ? 2 : 1;   // V_j travels with K_{j+lag} (2 in split-KV mode)
       const bool textq = ((wi.w >> 25) & 1) != 0;   // the queries are text tokens: every key is attended
       const int head_ld = prm.shared_qkv ? 0 : head;   // head coordinate of the q, k, v loads
@@ -656,9 +676,13 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
             slab_shape(g, sub0 + i, et, eh, ew, ntok, last);
           }
           const uint32_t dst = sbase + kOffQ + (uint32_t)i * kSlabBytes;
-          mbar_expect_tx(bar(kBarQFull + i), (uint32_t)ntok * 256u);
-          tma_load_5d(dst, &tms.q[last], bar(kBarQFull + i), 0, w0, h0, t0, head_ld);
-          tma_load_5d(dst + kHalfBytes, &tms.q[last], bar(kBarQFull + i), 64, w0, h0, t0, head_ld);
+          if (PSA_CHECKED(w0 >= 0 && h0 >= 0 && t0 >= 0 && head_ld >= 0 && head_ld < g.n_heads && last >= 0 && last <= 2 &&
+                          ntok > 0 && ntok <= kSlabTokens &&
+                          (textq || (w0 < g.Wp * g.bw && h0 < g.Hp * g.bh && t0 < g.Tp * g.bt)), 0xD01)) {   // inside the padded grid
+            mbar_expect_tx(bar(kBarQFull + i), (uint32_t)ntok * 256u);
+            tma_load_5d(dst, &tms.q[last], bar(kBarQFull + i), 0, w0, h0, t0, head_ld);
+            tma_load_5d(dst + kHalfBytes, &tms.q[last], bar(kBarQFull + i), 64, w0, h0, t0, head_ld);
+          }
         }
         if (i == 0) ++it_q0; else ++it_q1;
       }
@@ -681,7 +705,9 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
         }
         ok = mbar_wait_warp(bar(kBarSlotEmpty + k_slot), (k_use & 1u) ^ 1u, abort_flag, 0x110);
         if (!ok) return;
-        if (lane == 0) {
+        if (lane == 0 && PSA_CHECKED(v_slot < (uint32_t)kNumSlots && k_slot < (uint32_t)kNumSlots && t0 >= 0 && h0 >= 0 && w0 >= 0 &&
+                                     last >= 0 && last <= 2 && ntok > 0 && ntok <= kSlabTokens &&
+                                     (!with_v || (at0 >= 0 && ah0 >= 0 && aw0 >= 0 && alast >= 0 && alast <= 2)), 0xD02)) {
           uint32_t* m = meta + (kv_g % kMetaRing) * 8;
           m[0] = vw0; m[1] = vw1; m[2] = vw2; m[3] = vw3;
           const uint32_t pb = bar(kBarPairFull + pair_g % kNumPairBars);
@@ -756,7 +782,8 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
         const uint32_t v_slot = tile_g % kNumSlots, v_use = tile_g / kNumSlots;
         ok = mbar_wait_warp(bar(kBarSlotEmpty + v_slot), (v_use & 1u) ^ 1u, abort_flag, 0x112);
         if (!ok) break;
-        if (lane == 0) {
+        if (lane == 0 && PSA_CHECKED(v_slot < (uint32_t)kNumSlots && at0 >= 0 && ah0 >= 0 && aw0 >= 0 && alast >= 0 && alast <= 2 &&
+                                     antok > 0 && antok <= kSlabTokens, 0xD03)) {
           const uint32_t pb = bar(kBarPairFull + pair_g % kNumPairBars);
           mbar_expect_tx(pb, (uint32_t)antok * 256u);
           const uint32_t dv = sbase + kOffRing + v_slot * kSlabBytes;
@@ -811,6 +838,8 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
     // nk = keys of the slab (N of the instruction): 128, or fewer for a block's last slab.
     // iq: Q buffer; it: S tile written (they differ only in split-KV items).
     auto issue_qk = [&](int iq, uint32_t kslot, int nk, int it) {
+      if (!PSA_CHECKED(iq >= 0 && iq < 2 && it >= 0 && it < 2 && kslot < (uint32_t)kNumSlots && nk >= 16 && nk <= 128 && (nk & 15) == 0, 0xD20))
+        return;
       const uint32_t a0 = q_lo + (uint32_t)iq * kSlabStep, b0 = ring_lo_k + kslot * kSlabStep;
       const uint32_t idesc = instr_desc(false, (uint32_t)nk);
 #pragma unroll
@@ -824,6 +853,7 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
     // 16 keys advance 2048 bytes, the second 64 columns of head_dim sit one half slab
     // further (leading byte offset).
     auto issue_pv_half = [&](int i, uint32_t vslot, int half, bool accumulate, int nk) {
+      if (!PSA_CHECKED(i >= 0 && i < 2 && half >= 0 && half < 2 && vslot < (uint32_t)kNumSlots && nk >= 16 && nk <= 128, 0xD21)) return;
       const uint32_t b0 = ring_lo_v + vslot * kSlabStep;
 #pragma unroll
       for (int k4 = 0; k4 < 4; ++k4) {
@@ -1150,7 +1180,9 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
           const int col = c4 * 32 + c8 * 8;
           const int half = col >> 6, chunk = (col & 63) >> 3;
           uint8_t* dst = stage + half * kHalfBytes + row * 128 + ((chunk ^ (row & 7)) << 4);
-          *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
+          if (PSA_CHECKED(dst >= smem + kOffQ && dst + 16 <= smem + kOffQ + 2u * kSlabBytes &&
+                          (reinterpret_cast<uintptr_t>(dst) & 15u) == 0u, 0xD12))
+            *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
         }
       }
       tc_fence_before();
@@ -1160,7 +1192,8 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
       const float lse_row = empty ? neg_inf : (m_ref + log2f(l)) * 0.6931471805599453f;
       if (textq) {   // text slab: rows are consecutive text tokens; they follow the L video tokens
         t0 = 0; h0 = 0; w0 = (sub0 + qi) * kSlabTokens; last = 2;
-        if (w0 + row < g.n_text) prm.lse[(long long)head * g.Lt + g.L + w0 + row] = lse_row;
+        if (w0 + row < g.n_text && PSA_CHECKED(head >= 0 && head < g.n_heads && w0 >= 0, 0xD10))
+          prm.lse[(long long)head * g.Lt + g.L + w0 + row] = lse_row;
       } else {
         slab_origin(g, qb, sub0 + qi, t0, h0, w0);
         slab_shape(g, sub0 + qi, et, eh, ew, ntok, last);
@@ -1168,7 +1201,7 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
         const int t = t0 + ti_, hh = h0 + hi_, ww = w0 + wi_;
         if (row < ntok && t < g.T && hh < g.H && ww < g.W) {
           const long long tok = ((long long)t * g.H + hh) * g.W + ww;
-          prm.lse[(long long)head * g.Lt + tok] = lse_row;
+          if (PSA_CHECKED(head >= 0 && head < g.n_heads && tok >= 0 && tok < g.L, 0xD11)) prm.lse[(long long)head * g.Lt + tok] = lse_row;
         }
       }
       // Every thread's staged row is made visible to the TMA engine; the warpgroup's first warp
@@ -1180,8 +1213,10 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
         if (!ok) break;
         if (lane == 0) {
           const uint32_t src = sbase + kOffQ + (uint32_t)qi * kSlabBytes;
-          tma_store_5d(&tms.o[last], src, 0, w0, h0, t0, head);
-          tma_store_5d(&tms.o[last], src + kHalfBytes, 64, w0, h0, t0, head);
+          if (PSA_CHECKED(w0 >= 0 && h0 >= 0 && t0 >= 0 && head >= 0 && head < g.n_heads && last >= 0 && last <= 2, 0xD13)) {
+            tma_store_5d(&tms.o[last], src, 0, w0, h0, t0, head);
+            tma_store_5d(&tms.o[last], src + kHalfBytes, 64, w0, h0, t0, head);
+          }
           tma_store_commit();
           tma_store_wait_read();
           mbar_arrive(bar(kBarQEmpty + qi));

@@ -315,6 +315,7 @@ const char* psa_status_string(int status) {
     case PSA_ERR_CAPACITY: return "capacity exceeded (col_idx too small, or problem beyond the fixed scratch)";
     case PSA_ERR_CUDA: return "CUDA call failed";
     case PSA_ERR_TIMEOUT: return "device-side wait timed out";
+    case PSA_ERR_INTERNAL: return "kernel-side consistency check failed (checked build)";
     default: return "unknown status";
   }
 }

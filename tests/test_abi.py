@@ -34,7 +34,7 @@ def test_exports_every_declared_symbol(B):
 
 def test_status_strings(B):
     assert B.status_string(0) == "ok"
-    for code in (-1, -2, -3, -4, -5):
+    for code in (-1, -2, -3, -4, -5, -6):
         assert B.status_string(code) not in ("ok", "unknown status")
     assert B.status_string(-99) == "unknown status"
 
