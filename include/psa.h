@@ -26,7 +26,10 @@
  *     or aborted.
  *   - The library keeps one lazily created device workspace per device (work order,
  *     status word); calls that overlap on the GPU from different streams race on it.
- *     psa_shutdown() frees it.
+ *     psa_shutdown() frees it.  Once a call has sized that workspace, psa_mask_build and
+ *     psa_attn_fwd of the same or a smaller problem allocate nothing and synchronise nothing:
+ *     they can be captured in a CUDA graph and replayed (all arguments are captured by value;
+ *     the buffers' contents may change between replays).
  */
 #ifndef PSA_H_
 #define PSA_H_

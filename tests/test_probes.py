@@ -153,3 +153,45 @@ def test_scores_growing_along_the_keys_force_rescales(B, tile):
         err = np.abs(out_h[hd] - ro)
         assert err.max() <= 2e-2 and err.mean() <= 2e-3, (hd, err.max(), err.mean())
         assert np.abs(lse_h[hd] - rl).max() <= 1e-3, (hd, np.abs(lse_h[hd] - rl).max(), np.abs(rl).max())
+
+
+def test_forward_call_replays_from_a_cuda_graph(B):
+    """After a first call (which sizes the cached workspace) psa_mask_build + psa_attn_fwd allocate nothing
+    and synchronise nothing, so a step can be captured in a CUDA graph and replayed: the replay must see
+    new contents of the same buffers and give, bit for bit, what direct calls give."""
+    grid, tile = (4, 30, 32), (1, 15, 16)
+    params = [(2, 0, INF, 2, 0, 3), (1, 1, 2, 3, 0, INF), (4, 0, INF, 1, -1, INF)]
+    T, H, W = grid
+    L, nh = T * H * W, len(params)
+    bits = [{n: WL.tensor_bits(0x95 + i, n, nh, L) for n in ("q", "k", "v")} for i in range(2)]
+    dev = [{n: torch.from_numpy(b[n].view(np.int16)).cuda().view(torch.bfloat16) for n in b} for b in bits]
+    direct = [B.psa_attn_fwd(d["q"], d["k"], d["v"], params, grid, tile, SCALE) for d in dev]
+    assert B.psa_last_device_status()[0] == 0
+    q, k, v = (torch.empty_like(dev[0][n]) for n in ("q", "k", "v"))
+    out, lse = torch.empty_like(q), torch.empty((nh, L), dtype=torch.float32, device="cuda")
+    nb, nnz = B.psa_mask_sizes(params, grid, tile)
+    mask_out = (torch.empty((nh, nb, nb), dtype=torch.uint8, device="cuda"),
+                torch.empty(nh * nb + 1, dtype=torch.int32, device="cuda"),
+                torch.empty(max(nnz, 1), dtype=torch.int32, device="cuda"))
+    stream = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        B.psa_attn_fwd(q, k, v, params, grid, tile, SCALE, out=out, lse=lse, stream=stream)   # warm-up on this stream
+        torch.cuda.synchronize()
+        graph.capture_begin()
+        B.psa_mask_build(params, grid, tile, out=mask_out, stream=stream)
+        B.psa_attn_fwd(q, k, v, params, grid, tile, SCALE, out=out, lse=lse, stream=stream)
+        graph.capture_end()
+    ref_mask = B.psa_mask_build(params, grid, tile)
+    for i in (0, 1, 0):
+        for n, t in (("q", q), ("k", k), ("v", v)):
+            t.copy_(dev[i][n])
+        out.fill_(float("nan"))
+        mask_out[0].fill_(255)
+        torch.cuda.synchronize()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(out.view(torch.int16), direct[i][0].view(torch.int16))
+        assert torch.equal(lse.view(torch.int32), direct[i][1].view(torch.int32))
+        assert all(torch.equal(a, b) for a, b in zip(mask_out, ref_mask))
+    assert B.psa_last_device_status()[0] == 0
