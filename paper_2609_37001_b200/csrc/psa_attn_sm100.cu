@@ -45,6 +45,11 @@ constexpr int kWarpMma = 0, kWarpLoad = 1, kUtilGroup = 0, kFirstSoftmaxWarp = 4
 constexpr int kNumSlots = 5;                       // K/V ring slots of one 128 x 128 bf16 slab
 constexpr uint32_t kSlabBytes = 128 * 128 * 2;     // 32 KB
 constexpr uint32_t kHalfBytes = kSlabBytes / 2;    // one 64-column swizzled half
+// Register budgets after the re-split (setmaxnreg).  The CTA's pool is what it was launched with
+// (kRegsAtLaunch per thread: the compiler's figure under the launch bound of 384 threads);
+// setmaxnreg.inc blocks until the pool has room, so a split that does not fit would never start.
+constexpr int kRegsAtLaunch = 168, kRegsUtil = 72, kRegsSoftmax = 216;
+static_assert(128 * kRegsUtil + 256 * kRegsSoftmax <= kThreads * kRegsAtLaunch, "register re-split exceeds the CTA's pool");
 constexpr int kMetaRing = 8;
 constexpr float kRescaleThreshold = 8.0f;          // log2 units; lazy rescale of O
 constexpr unsigned long long kTimeoutNs = 2000000000ull;
@@ -610,7 +615,7 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
 
   if ((warp >> 2) == kUtilGroup) {
   // Utility warpgroup: give registers away (the budget is re-split per warpgroup).
-  asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
+  asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsUtil));
   if (warp == kWarpLoad) {
     // ======================================================================= load warp
     // Ring tiles are issued in the order K_0, V_0, K_1, V_1, ...; the MMA warp needs V_j and
@@ -1058,7 +1063,7 @@ attn_fwd_kernel(const __grid_constant__ TensorMaps tms, const AttnParams prm) {
     __syncwarp();
   }
   } else {
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmax));
     // ======================================================================= softmax warps
     const int qi = (warp - kFirstSoftmaxWarp) >> 2;   // tile (S_i, O_i) handled by this warpgroup
     const int row = (warp & 3) * 32 + lane;       // row of the slab == TMEM lane
