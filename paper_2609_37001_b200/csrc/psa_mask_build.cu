@@ -1,7 +1,7 @@
 // psa_mask_build: block mask and GetKVBlocks index lists from the stripe parameters
 // (Algorithm 1 evaluated on block coordinates; Algorithm 2, producer side).
-// Integer work only.  Two kernels: a register-only one for block grids of at most 32 x 32
-// coordinates per axis pair (mask_build_small_kernel, further down), and the general one
+// Integer work only.  Two kernels: a register-only one for block grids of at most 64 temporal x 32 spatial
+// coordinates (mask_build_small_kernel, further down), and the general one
 // described here.
 //
 // The two conditions of Algorithm 1 depend only on coordinate differences, so each block of
@@ -130,17 +130,17 @@ mask_build_kernel(const HeadParamsArray hp, const HeadBases hb, const Geom g, in
     row_ptr[(long long)n_heads_here * g.NB] = total_nnz;
 }
 
-// Fast path for block grids with at most 32 temporal and 32 spatial block coordinates (all the
+// Fast path for block grids with at most 64 temporal and 32 spatial block coordinates (all the
 // paper's shapes): no shared-memory tables and no block-wide barrier.  The host evaluates the
 // two axis conditions of Algorithm 1 once per head for every coordinate difference and hands
-// the kernel two 64-bit sets per head (bit d + n - 1 of an axis' set = "difference d attends"),
+// the kernel two bit sets per head (127 and 63 bits) (bit d + n - 1 of an axis' set = "difference d attends"),
 // so the key coordinates a query coordinate x attends are one shift away:
 // (set >> (n - 1 - x)) & ((1 << n) - 1).  Row counts are popcounts, their prefix sums one warp
 // scan.  A warp then owns whole rows: the byte mask is written 32 key blocks per step, and the
 // column list -- the sorted Cartesian product of the two attended coordinate sets -- 32
 // consecutive entries per step.
 struct HeadSets {
-  unsigned long long setT[kMaxHeads], setS[kMaxHeads];
+  unsigned long long setT[kMaxHeads], setT_hi[kMaxHeads], setS[kMaxHeads];   // temporal set: 127 bits
   int base[kMaxHeads];  // number of attended block pairs of all earlier heads
 };
 
@@ -156,22 +156,32 @@ mask_build_small_kernel(const HeadSets hs, const Geom g, int n_heads_here, int r
   const int q0 = (blockIdx.x * nwarps + warp) * rows_per_warp;
   const int q1 = min(g.NB, q0 + rows_per_warp);
   if (q0 >= q1) return;
-  const unsigned long long setT = hs.setT[h], setS = hs.setS[h];
-  const unsigned maskT = Tp == 32 ? 0xffffffffu : ((1u << Tp) - 1u), maskS = Sp == 32 ? 0xffffffffu : ((1u << Sp) - 1u);
-  auto rowT = [&](int x) -> unsigned { return (unsigned)(setT >> (Tp - 1 - x)) & maskT; };
+  const unsigned long long setT = hs.setT[h], setT_hi = hs.setT_hi[h], setS = hs.setS[h];
+  const unsigned long long maskT = Tp == 64 ? ~0ull : ((1ull << Tp) - 1ull);
+  const unsigned maskS = Sp == 32 ? 0xffffffffu : ((1u << Sp) - 1u);
+  // temporal key coordinates attended by query coordinate x (up to 64 of them: a 64-bit mask)
+  auto rowT = [&](int x) -> unsigned long long {
+    const int sh = Tp - 1 - x;   // 0 .. 63
+    const unsigned long long lo = setT >> sh, hi = sh ? (setT_hi << (64 - sh)) : 0ull;
+    return (lo | hi) & maskT;
+  };
   auto rowS = [&](int x) -> unsigned { return (unsigned)(setS >> (Sp - 1 - x)) & maskS; };
-  // lane x holds the count of coordinate x and the exclusive prefix of the counts before it
-  const int cntT = lane < Tp ? __popc(rowT(lane)) : 0, cntS = lane < Sp ? __popc(rowS(lane)) : 0;
-  int incT = cntT, incS = cntS;
+  // lane x holds the counts of coordinates x (and x + 32 on the temporal axis) and the exclusive
+  // prefixes of the counts before them
+  const int cntT0 = lane < Tp ? __popcll(rowT(lane)) : 0, cntT1 = lane + 32 < Tp ? __popcll(rowT(lane + 32)) : 0;
+  const int cntS = lane < Sp ? __popc(rowS(lane)) : 0;
+  int incT0 = cntT0, incT1 = cntT1, incS = cntS;
 #pragma unroll
   for (int off = 1; off < 32; off <<= 1) {
-    const int a = __shfl_up_sync(0xffffffffu, incT, off), b = __shfl_up_sync(0xffffffffu, incS, off);
-    if (lane >= off) { incT += a; incS += b; }
+    const int a = __shfl_up_sync(0xffffffffu, incT0, off), c = __shfl_up_sync(0xffffffffu, incT1, off);
+    const int b = __shfl_up_sync(0xffffffffu, incS, off);
+    if (lane >= off) { incT0 += a; incT1 += c; incS += b; }
   }
-  const int preT = incT - cntT, preS = incS - cntS;
+  const int sumT0 = __shfl_sync(0xffffffffu, incT0, 31);
+  const int preT0 = incT0 - cntT0, preT1 = sumT0 + incT1 - cntT1, preS = incS - cntS;
   const int sumS = __shfl_sync(0xffffffffu, incS, 31);
-  __shared__ int strips[8 * 64];           // per warp: the r-th attended temporal / spatial coordinate
-  int* strip = strips + warp * 64;
+  __shared__ int strips[8 * 96];           // per warp: the r-th attended temporal (64) / spatial (32) coordinate
+  int* strip = strips + warp * 96;
   int tq_tab = -1;                         // query coordinate the temporal table was built for
   const unsigned lane_lt = (1u << lane) - 1u;
   // coordinates of key block `lane`, and the advance of 32 key blocks
@@ -181,15 +191,17 @@ mask_build_small_kernel(const HeadSets hs, const Geom g, int n_heads_here, int r
   uint8_t* mrow = block_mask ? block_mask + ((long long)h * g.NB + q0) * g.NB : nullptr;
   int* rp = row_ptr ? row_ptr + (long long)h * g.NB + q0 : nullptr;
   for (int qb = q0; qb < q1; ++qb) {
-    const unsigned mT = rowT(tq), mS = rowS(sq);
-    const int cT = __shfl_sync(0xffffffffu, cntT, tq), pT = __shfl_sync(0xffffffffu, preT, tq);
+    const unsigned long long mT = rowT(tq);
+    const unsigned mS = rowS(sq);
+    const int cT = __shfl_sync(0xffffffffu, tq < 32 ? cntT0 : cntT1, tq & 31);
+    const int pT = __shfl_sync(0xffffffffu, tq < 32 ? preT0 : preT1, tq & 31);
     const int cS = __shfl_sync(0xffffffffu, cntS, sq), pS = __shfl_sync(0xffffffffu, preS, sq);
     const int pos = hs.base[h] + pT * sumS + cT * pS;
     if (rp && lane == 0) *rp = pos;
     if (mrow) {
       int tk = tk0, sk = sk0;
       for (int kb = lane; kb < g.NB; kb += 32) {
-        mrow[kb] = (uint8_t)(((mT >> tk) & (mS >> sk)) & 1u);
+        mrow[kb] = (uint8_t)(((unsigned)(mT >> tk) & (mS >> sk)) & 1u);
         tk += dt;
         sk += ds;
         if (sk >= Sp) { sk -= Sp; ++tk; }
@@ -198,21 +210,22 @@ mask_build_small_kernel(const HeadSets hs, const Geom g, int n_heads_here, int r
     }
     if (col_idx && cT * cS > 0) {
       // Entry e of the row's list is (the (e / cS)-th attended temporal coordinate, the
-      // (e % cS)-th attended spatial one).  "The r-th set bit" comes from two 32-entry tables in the
-      // warp's strip (a lane whose bit is set writes its index at its rank; the temporal table
-      // only changes with tq); e / cS is a multiply and a shift (e < 1024, cS <= 32).  The list is
-      // then written 32 consecutive entries per store.
+      // (e % cS)-th attended spatial one).  "The r-th set bit" comes from two tables in the warp's
+      // strip (a lane whose bit is set writes its index at its rank; the temporal table only
+      // changes with tq); e / cS is a multiply and a shift (e < 2048, cS <= 32).  The list is then
+      // written 32 consecutive entries per store.
       if (tq != tq_tab) {
-        if ((mT >> lane) & 1u) strip[__popc(mT & lane_lt)] = lane;
+        if ((mT >> lane) & 1ull) strip[__popcll(mT & (unsigned long long)lane_lt)] = lane;
+        if ((mT >> (lane + 32)) & 1ull) strip[__popcll(mT & ((1ull << (lane + 32)) - 1ull))] = lane + 32;
         tq_tab = tq;
       }
-      if ((mS >> lane) & 1u) strip[32 + __popc(mS & lane_lt)] = lane;
+      if ((mS >> lane) & 1u) strip[64 + __popc(mS & lane_lt)] = lane;
       __syncwarp();
       const int count = cT * cS;
-      const unsigned inv = (65536u + (unsigned)cS - 1u) / (unsigned)cS;
+      const unsigned inv = ((1u << 20) + (unsigned)cS - 1u) / (unsigned)cS;
       for (int e = lane; e < count; e += 32) {
-        const int it = (int)(((unsigned)e * inv) >> 16), is = e - it * cS;
-        col_idx[pos + e] = strip[it] * Sp + strip[32 + is];
+        const int it = (int)(((unsigned)e * inv) >> 20), is = e - it * cS;
+        col_idx[pos + e] = strip[it] * Sp + strip[64 + is];
       }
       __syncwarp();
     }
@@ -226,18 +239,19 @@ cudaError_t launch_mask_build(const HeadParamsArray& hp, const int* head_bases, 
                               int n_sms, cudaStream_t stream, int* launches) {
   HeadBases hb;
   for (int h = 0; h < kMaxHeads; ++h) hb.base[h] = h < n_heads_here ? head_bases[h] : 0;
-  if (g.Tp <= 32 && g.Sp <= 32) {
+  if (g.Tp <= 64 && g.Sp <= 32) {
     HeadSets hs;
     for (int h = 0; h < kMaxHeads; ++h) {
-      unsigned long long st = 0, ss = 0;
+      unsigned long long st = 0, st_hi = 0, ss = 0;
       if (h < n_heads_here) {
         const psa_head_params& p = hp.p[h];
         for (int i = 0; i < 2 * g.Tp - 1; ++i)
-          if (axis_attends(i - (g.Tp - 1), p.Tw, p.To, p.Ts)) st |= 1ull << i;
+          if (axis_attends(i - (g.Tp - 1), p.Tw, p.To, p.Ts)) (i < 64 ? st : st_hi) |= 1ull << (i & 63);
         for (int i = 0; i < 2 * g.Sp - 1; ++i)
           if (axis_attends(i - (g.Sp - 1), p.Sw, p.So, p.Ss)) ss |= 1ull << i;
       }
       hs.setT[h] = st;
+      hs.setT_hi[h] = st_hi;
       hs.setS[h] = ss;
       hs.base[h] = h < n_heads_here ? head_bases[h] : 0;
     }
