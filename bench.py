@@ -754,7 +754,7 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="wan14b_720p")
+    ap.add_argument("--workload", default="wan14b_720p", help="a name from workloads.json, or 'all' (= the default run: headline + configs array)")
     ap.add_argument("--quick", action="store_true", help="timed region only (no dense/e2e/CPU legs); for profiling")
     ap.add_argument("--no-configs", action="store_true", help="skip the kernel-level timing of the other configurations")
     ap.add_argument("--ulysses", action="store_true",
@@ -777,6 +777,8 @@ def main():
         run_report(args)
         return
     from paper_2609_37001_b200 import workloads as WL
+    if args.workload == "all":      # the default run already is "all": headline line + the `configs` array
+        args.workload, args.no_configs = "wan14b_720p", False
     w = WL.workload(args.workload)
     if args.impl == "reference":
         run_reference(args, w)
