@@ -38,7 +38,7 @@ SCALE = 1.0 / math.sqrt(128.0)
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 DATASHEET_BF16_TFLOPS = 2250.0   # nominal dense bf16 figure of the part (context beside the measured peak)
 # the other configurations of the benchmark set, timed at kernel level after the headline
-OTHER_CONFIGS = ["tiny", "wan13b_480p", "wan13b_480p_b3x32x4", "hunyuan_720p", "sweep_00", "sweep_25", "sweep_50", "sweep_75", "sweep_90",
+OTHER_CONFIGS = ["tiny", "wan13b_480p", "wan13b_480p_b3x32x4", "wan13b_480p_b1x30x8", "wan13b_480p_b1x32x4", "hunyuan_720p", "sweep_00", "sweep_25", "sweep_50", "sweep_75", "sweep_90",
                  "ragged_75", "wan14b_720p_b3x8x16", "hunyuan_768p"]
 
 

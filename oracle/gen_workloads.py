@@ -98,6 +98,12 @@ def main():
     rng = np.random.Generator(np.random.Philox(key=0x50534102))
     wl.append(describe("wan13b_480p_b3x32x4", grid, tile, draw_heads(rng, candidates(*grid, tile), 12, 0.50, 0.80),
                        "12 heads, 50-80% tile sparsity, temporal/spatial/joint in turn", 0x50534102))
+    #    and with blocks that pad only W: 1x30x8 (240 tokens = a 128- and a 112-token slab, W 52 -> 56) and
+    #    the 128-token 1x32x4 (H 30 -> 32)
+    for name, tile in (("wan13b_480p_b1x30x8", (1, 30, 8)), ("wan13b_480p_b1x32x4", (1, 32, 4))):
+        rng = np.random.Generator(np.random.Philox(key=0x50534102))
+        wl.append(describe(name, grid, tile, draw_heads(rng, candidates(*grid, tile), 12, 0.50, 0.80),
+                           "12 heads, 50-80% tile sparsity, temporal/spatial/joint in turn", 0x50534102))
     # 3. Wan 2.1 14B 720p (headline).  1x15x16 (240 tokens = a 128- and a 112-token slab) tiles 21x45x80
     #    exactly; 1x16x16 and the paper's 3x8x16 pad H to 48 and are kept as further test cases.
     grid = (21, 45, 80)

@@ -164,6 +164,8 @@ def _sampled_rows(grid, tile, seed):
 @pytest.mark.parametrize("name,heads", [
     ("wan13b_480p", None),
     ("wan13b_480p_b3x32x4", [0, 4, 7, 11]),
+    ("wan13b_480p_b1x30x8", [1, 5, 8, 10]),
+    ("wan13b_480p_b1x32x4", [2, 6, 9]),
     ("wan14b_720p", list(range(0, 40, 5))),
     ("wan14b_720p_b1x16x16", [2, 17, 31]),
     ("wan14b_720p_b3x8x16", [0, 13, 26]),
