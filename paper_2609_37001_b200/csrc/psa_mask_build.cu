@@ -1,8 +1,8 @@
 // psa_mask_build: block mask and GetKVBlocks index lists from the stripe parameters
 // (Algorithm 1 evaluated on block coordinates; Algorithm 2, producer side).
-// Integer work only.  Two kernels: a register-only one for block grids of at most 64 temporal x 32 spatial
-// coordinates (mask_build_small_kernel, further down), and the general one
-// described here.
+// Integer work only.  Two kernels: one for block grids of at most 64 temporal x 32 spatial
+// coordinates (mask_build_small_kernel, further down: one thread block per head and temporal
+// query coordinate), and the general one described here.
 //
 // The two conditions of Algorithm 1 depend only on coordinate differences, so each block of
 // threads first tabulates, for its head, "does difference d attend" for every temporal and
@@ -131,31 +131,41 @@ mask_build_kernel(const HeadParamsArray hp, const HeadBases hb, const Geom g, in
 }
 
 // Fast path for block grids with at most 64 temporal and 32 spatial block coordinates (all the
-// paper's shapes): no shared-memory tables and no block-wide barrier.  The host evaluates the
-// two axis conditions of Algorithm 1 once per head for every coordinate difference and hands
-// the kernel two bit sets per head (127 and 63 bits) (bit d + n - 1 of an axis' set = "difference d attends"),
-// so the key coordinates a query coordinate x attends are one shift away:
-// (set >> (n - 1 - x)) & ((1 << n) - 1).  Row counts are popcounts, their prefix sums one warp
-// scan.  A warp then owns whole rows: the byte mask is written 32 key blocks per step, and the
-// column list -- the sorted Cartesian product of the two attended coordinate sets -- 32
-// consecutive entries per step.
+// paper's shapes): no block-wide table building.  The host evaluates the two axis conditions of
+// Algorithm 1 once per head for every coordinate difference and hands the kernel two bit sets
+// per head (127 and 63 bits; bit d + n - 1 of an axis' set = "difference d attends"), so the key
+// coordinates a query coordinate x attends are one shift away: (set >> (n - 1 - x)) & ((1 << n) - 1).
+//
+// One thread block per (head, temporal query coordinate tq): its S' rows are consecutive, so
+// their mask bytes are one contiguous region and their column lists one contiguous range.
+//   * Warp 0 derives the row counts (popcounts), their prefix sums (one warp scan), the block's
+//     first list offset, "the r-th attended temporal coordinate" of tq, and writes the S' row
+//     offsets.
+//   * Meanwhile all threads write the mask region 32 bytes at a time: a thread assembles 32
+//     consecutive mask bits (the row of the Kronecker product is the spatial bit pattern repeated
+//     under the temporal bits), spreads them to bytes with four multiplies per 16 and stores two
+//     16-byte words.
+//   * After one barrier the rows of the block are taken by sub-groups of 8, 16 or 32 lanes: entry e
+//     of a row's list is (the (e / cS)-th attended temporal coordinate, the (e % cS)-th attended
+//     spatial one); the division is a multiply and a shift (e < 2048, cS <= 32).
 struct HeadSets {
   unsigned long long setT[kMaxHeads], setT_hi[kMaxHeads], setS[kMaxHeads];   // temporal set: 127 bits
   int base[kMaxHeads];  // number of attended block pairs of all earlier heads
 };
 
+// n / d for n < 2^16, d <= 2^11 with m = ceil(2^40 / d): exact (n * (m * d - 2^40) < 2^40)
+__device__ __forceinline__ int div_magic(int n, unsigned long long m) { return (int)(((unsigned long long)(unsigned)n * m) >> 40); }
+
 __global__ void __launch_bounds__(256)
-mask_build_small_kernel(const HeadSets hs, const Geom g, int n_heads_here, int rows_per_warp,
-                        uint8_t* __restrict__ block_mask, int* __restrict__ row_ptr, int* __restrict__ col_idx,
-                        int total_nnz) {
-  const int h = blockIdx.y;
+mask_build_small_kernel(const HeadSets hs, const Geom g, int n_heads_here, unsigned long long magic_nb,
+                        unsigned long long magic_sp, uint8_t* __restrict__ block_mask, int* __restrict__ row_ptr,
+                        int* __restrict__ col_idx, int total_nnz) {
+  const int h = blockIdx.y, tq = blockIdx.x;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
-  const int Tp = g.Tp, Sp = g.Sp;
-  if (row_ptr && blockIdx.x == 0 && h == n_heads_here - 1 && threadIdx.x == 0)
-    row_ptr[(long long)n_heads_here * g.NB] = total_nnz;
-  const int q0 = (blockIdx.x * nwarps + warp) * rows_per_warp;
-  const int q1 = min(g.NB, q0 + rows_per_warp);
-  if (q0 >= q1) return;
+  const int Tp = g.Tp, Sp = g.Sp, NB = g.NB;
+  __shared__ int s_preS[32], s_cS[32], s_tsel[64], s_hdr[2];
+  __shared__ int s_strip[8 * 4 * 32];      // per warp and sub-group: the r-th attended spatial coordinate of its row
+  __shared__ unsigned s_inv[33];           // ceil(2^20 / c): e / c = (e * inv) >> 20 for e < 2048, c <= 32
   const unsigned long long setT = hs.setT[h], setT_hi = hs.setT_hi[h], setS = hs.setS[h];
   const unsigned long long maskT = Tp == 64 ? ~0ull : ((1ull << Tp) - 1ull);
   const unsigned maskS = Sp == 32 ? 0xffffffffu : ((1u << Sp) - 1u);
@@ -166,71 +176,134 @@ mask_build_small_kernel(const HeadSets hs, const Geom g, int n_heads_here, int r
     return (lo | hi) & maskT;
   };
   auto rowS = [&](int x) -> unsigned { return (unsigned)(setS >> (Sp - 1 - x)) & maskS; };
-  // lane x holds the counts of coordinates x (and x + 32 on the temporal axis) and the exclusive
-  // prefixes of the counts before them
-  const int cntT0 = lane < Tp ? __popcll(rowT(lane)) : 0, cntT1 = lane + 32 < Tp ? __popcll(rowT(lane + 32)) : 0;
-  const int cntS = lane < Sp ? __popc(rowS(lane)) : 0;
-  int incT0 = cntT0, incT1 = cntT1, incS = cntS;
-#pragma unroll
-  for (int off = 1; off < 32; off <<= 1) {
-    const int a = __shfl_up_sync(0xffffffffu, incT0, off), c = __shfl_up_sync(0xffffffffu, incT1, off);
-    const int b = __shfl_up_sync(0xffffffffu, incS, off);
-    if (lane >= off) { incT0 += a; incT1 += c; incS += b; }
-  }
-  const int sumT0 = __shfl_sync(0xffffffffu, incT0, 31);
-  const int preT0 = incT0 - cntT0, preT1 = sumT0 + incT1 - cntT1, preS = incS - cntS;
-  const int sumS = __shfl_sync(0xffffffffu, incS, 31);
-  __shared__ int strips[8 * 96];           // per warp: the r-th attended temporal (64) / spatial (32) coordinate
-  int* strip = strips + warp * 96;
-  int tq_tab = -1;                         // query coordinate the temporal table was built for
+  const unsigned long long mT = rowT(tq);
   const unsigned lane_lt = (1u << lane) - 1u;
-  // coordinates of key block `lane`, and the advance of 32 key blocks
-  const int tk0 = lane / Sp, sk0 = lane - tk0 * Sp;
-  const int dt = 32 / Sp, ds = 32 - dt * Sp;
-  int tq = q0 / Sp, sq = q0 - tq * Sp;
-  uint8_t* mrow = block_mask ? block_mask + ((long long)h * g.NB + q0) * g.NB : nullptr;
-  int* rp = row_ptr ? row_ptr + (long long)h * g.NB + q0 : nullptr;
-  for (int qb = q0; qb < q1; ++qb) {
-    const unsigned long long mT = rowT(tq);
-    const unsigned mS = rowS(sq);
-    const int cT = __shfl_sync(0xffffffffu, tq < 32 ? cntT0 : cntT1, tq & 31);
-    const int pT = __shfl_sync(0xffffffffu, tq < 32 ? preT0 : preT1, tq & 31);
-    const int cS = __shfl_sync(0xffffffffu, cntS, sq), pS = __shfl_sync(0xffffffffu, preS, sq);
-    const int pos = hs.base[h] + pT * sumS + cT * pS;
-    if (rp && lane == 0) *rp = pos;
-    if (mrow) {
-      int tk = tk0, sk = sk0;
-      for (int kb = lane; kb < g.NB; kb += 32) {
-        mrow[kb] = (uint8_t)(((unsigned)(mT >> tk) & (mS >> sk)) & 1u);
-        tk += dt;
-        sk += ds;
-        if (sk >= Sp) { sk -= Sp; ++tk; }
-      }
-      mrow += g.NB;
+
+  if (threadIdx.x >= 64 && threadIdx.x <= 96) {
+    const unsigned c = threadIdx.x - 64;
+    s_inv[c] = c ? ((1u << 20) + c - 1u) / c : 0u;
+  }
+  if (warp == 0) {
+    // lane x holds the counts of coordinates x (and x + 32 on the temporal axis) and the exclusive
+    // prefixes of the counts before them
+    const int cntT0 = lane < Tp ? __popcll(rowT(lane)) : 0, cntT1 = lane + 32 < Tp ? __popcll(rowT(lane + 32)) : 0;
+    const int cntS = lane < Sp ? __popc(rowS(lane)) : 0;
+    int incT0 = cntT0, incT1 = cntT1, incS = cntS;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const int a = __shfl_up_sync(0xffffffffu, incT0, off), c = __shfl_up_sync(0xffffffffu, incT1, off);
+      const int b = __shfl_up_sync(0xffffffffu, incS, off);
+      if (lane >= off) { incT0 += a; incT1 += c; incS += b; }
     }
-    if (col_idx && cT * cS > 0) {
-      // Entry e of the row's list is (the (e / cS)-th attended temporal coordinate, the
-      // (e % cS)-th attended spatial one).  "The r-th set bit" comes from two tables in the warp's
-      // strip (a lane whose bit is set writes its index at its rank; the temporal table only
-      // changes with tq); e / cS is a multiply and a shift (e < 2048, cS <= 32).  The list is then
-      // written 32 consecutive entries per store.
-      if (tq != tq_tab) {
-        if ((mT >> lane) & 1ull) strip[__popcll(mT & (unsigned long long)lane_lt)] = lane;
-        if ((mT >> (lane + 32)) & 1ull) strip[__popcll(mT & ((1ull << (lane + 32)) - 1ull))] = lane + 32;
-        tq_tab = tq;
+    const int sumT0 = __shfl_sync(0xffffffffu, incT0, 31);
+    const int preT0 = incT0 - cntT0, preT1 = sumT0 + incT1 - cntT1, preS = incS - cntS;
+    const int sumS = __shfl_sync(0xffffffffu, incS, 31);
+    const int cT = __popcll(mT);
+    const int pT = __shfl_sync(0xffffffffu, tq < 32 ? preT0 : preT1, tq & 31);
+    const int pos0 = hs.base[h] + pT * sumS;
+    s_preS[lane] = preS;
+    s_cS[lane] = cntS;
+    if ((mT >> lane) & 1ull) s_tsel[__popcll(mT & (unsigned long long)lane_lt)] = lane;
+    if ((mT >> (lane + 32)) & 1ull) s_tsel[__popcll(mT & ((1ull << (lane + 32)) - 1ull))] = lane + 32;
+    if (lane == 0) { s_hdr[0] = cT; s_hdr[1] = pos0; }
+    if (row_ptr) {
+      if (lane < Sp) row_ptr[(long long)h * NB + tq * Sp + lane] = pos0 + cT * preS;
+      if (tq == 0 && h == n_heads_here - 1 && lane == 0) row_ptr[(long long)n_heads_here * NB] = total_nnz;
+    }
+  }
+
+  if (block_mask) {
+    // The block writes the 32-byte aligned chunks that START inside its rows' region; its last chunk
+    // runs on into the next region (next tq, or the next head), whose own first chunk starts at the
+    // next aligned address.  Only the very first bytes of the whole mask (when its base is not
+    // aligned) and a clipped chunk at its very end are written bytewise.
+    const int len = Sp * NB;                                 // bytes of this block's rows
+    uint8_t* p0 = block_mask + ((long long)h * NB + (long long)tq * Sp) * NB;
+    const int lead = (int)((32u - (unsigned)(reinterpret_cast<uintptr_t>(p0) & 31u)) & 31u);   // first aligned offset
+    // up to `limit` mask bytes from region offset r on (bit i of the result = byte r + i); *got = bytes that exist
+    auto gen = [&](int r, int limit, int* got) -> unsigned {
+      int hh = h, tq_ = tq;
+      int sq = div_magic(r, magic_nb), kb = r - sq * NB;
+      int tk = div_magic(kb, magic_sp), sk = kb - tk * Sp;
+      unsigned long long sT = setT, sT_hi = setT_hi, sS = setS, mT_ = mT;
+      unsigned mS = (unsigned)(sS >> (Sp - 1 - sq)) & maskS;
+      unsigned bits = 0u;
+      int n = 0;
+      while (n < limit && hh < n_heads_here) {
+        const unsigned grp = ((mT_ >> tk) & 1ull) ? (mS >> sk) : 0u;   // Sp - sk key blocks of temporal group tk
+        int take = Sp - sk;
+        if (take > limit - n) take = limit - n;
+        bits |= (take >= 32 ? grp : (grp & ((1u << take) - 1u))) << n;
+        n += take;
+        sk += take;
+        if (sk == Sp) {
+          sk = 0;
+          if (++tk == Tp) {
+            tk = 0;
+            if (++sq == Sp) {   // rare: the chunk runs on into the next region
+              sq = 0;
+              if (++tq_ == Tp) {
+                tq_ = 0;
+                if (++hh < n_heads_here) { sT = hs.setT[hh]; sT_hi = hs.setT_hi[hh]; sS = hs.setS[hh]; }
+              }
+              const int sh = Tp - 1 - tq_;
+              mT_ = ((sT >> sh) | (sh ? (sT_hi << (64 - sh)) : 0ull)) & maskT;
+            }
+            mS = (unsigned)(sS >> (Sp - 1 - sq)) & maskS;
+          }
+        }
       }
-      if ((mS >> lane) & 1u) strip[64 + __popc(mS & lane_lt)] = lane;
+      *got = n;
+      return bits;
+    };
+    const int nchunks = len > lead ? (len - lead + 31) >> 5 : 0;
+    for (int c = threadIdx.x; c < nchunks; c += blockDim.x) {
+      const int r = lead + 32 * c;
+      int n;
+      const unsigned bits = gen(r, 32, &n);
+      if (n == 32) {
+        uint32_t w[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) w[k] = (((bits >> (4 * k)) & 15u) * 0x00204081u) & 0x01010101u;
+        uint4* dst = reinterpret_cast<uint4*>(p0 + r);
+        dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
+        dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
+      } else {
+        for (int i = 0; i < n; ++i) p0[r + i] = (uint8_t)((bits >> i) & 1u);   // the end of the whole mask
+      }
+    }
+    if (h == 0 && tq == 0 && lead > 0 && threadIdx.x == blockDim.x - 1) {   // unaligned start of the whole mask
+      int n;
+      const unsigned bits = gen(0, lead, &n);
+      for (int i = 0; i < n; ++i) p0[i] = (uint8_t)((bits >> i) & 1u);
+    }
+  }
+  __syncthreads();
+
+  if (col_idx) {
+    // Sub-groups of 8, 16 or 32 lanes take one row each, so that the S' rows of the block are
+    // all in flight at once (S' <= 8, 16, 32 with eight warps).
+    const int cT = s_hdr[0], pos0 = s_hdr[1];
+    const int lg = Sp > 16 ? 2 : (Sp > 8 ? 1 : 0);          // log2 of the sub-groups per warp
+    const int W = 32 >> lg, grp = lane >> (5 - lg), sl = lane & (W - 1);
+    int* strip = s_strip + ((warp << 2) + grp) * 32;         // the r-th attended spatial coordinate of the row
+    for (int sq0 = warp << lg; sq0 < Sp && cT > 0; sq0 += nwarps << lg) {
+      const int sq = sq0 + grp;
+      const bool act = sq < Sp;
+      const int cS = act ? s_cS[sq] : 0;
+      const int pos = pos0 + cT * (act ? s_preS[sq] : 0);
+      const unsigned mS = act ? rowS(sq) : 0u;
+      for (int b = sl; b < 32; b += W)
+        if ((mS >> b) & 1u) strip[__popc(mS & ((1u << b) - 1u))] = b;
       __syncwarp();
       const int count = cT * cS;
-      const unsigned inv = ((1u << 20) + (unsigned)cS - 1u) / (unsigned)cS;
-      for (int e = lane; e < count; e += 32) {
+      const unsigned inv = s_inv[cS];
+      for (int e = sl; e < count; e += W) {
         const int it = (int)(((unsigned)e * inv) >> 20), is = e - it * cS;
-        col_idx[pos + e] = strip[it] * Sp + strip[64 + is];
+        col_idx[pos + e] = s_tsel[it] * Sp + strip[is];
       }
       __syncwarp();
     }
-    if (rp) ++rp;
-    if (++sq == Sp) { sq = 0; ++tq; }
   }
 }
 
@@ -255,14 +328,12 @@ cudaError_t launch_mask_build(const HeadParamsArray& hp, const int* head_bases, 
       hs.setS[h] = ss;
       hs.base[h] = h < n_heads_here ? head_bases[h] : 0;
     }
-    // one to three rows per warp: the per-row work is a dependent chain, so more warps beat longer ones
-    const int warps_wanted = 8 * 8 * n_sms;
-    int rows_per_warp = (int)(((long long)g.NB * n_heads_here + warps_wanted - 1) / warps_wanted);
-    if (rows_per_warp < 1) rows_per_warp = 1;
-    const int rows_per_block = 8 * rows_per_warp;
-    dim3 grid((g.NB + rows_per_block - 1) / rows_per_block, n_heads_here);
+    const unsigned long long two40 = 1ull << 40;
+    const unsigned long long magic_nb = (two40 + (unsigned long long)g.NB - 1ull) / (unsigned long long)g.NB;
+    const unsigned long long magic_sp = (two40 + (unsigned long long)g.Sp - 1ull) / (unsigned long long)g.Sp;
+    dim3 grid(g.Tp, n_heads_here);   // one block per (head, temporal query coordinate)
     mask_build_small_kernel<<<grid, 256, 0, stream>>>(
-        hs, g, n_heads_here, rows_per_warp, block_mask, row_ptr, col_idx, total_nnz_through_chunk);
+        hs, g, n_heads_here, magic_nb, magic_sp, block_mask, row_ptr, col_idx, total_nnz_through_chunk);
     ++*launches;
     return cudaGetLastError();
   }

@@ -72,3 +72,31 @@ def test_capacity_error_and_optional_outputs(B):
     torch.cuda.synchronize()
     _, orp, _ = O.block_index_lists(params, *grid, tile)
     assert np.array_equal(rp.cpu().numpy(), orp)
+
+
+@pytest.mark.parametrize("grid,tile,nh", [((4, 4, 4), (1, 1, 1), 3), ((3, 2, 2), (1, 1, 1), 5), ((5, 1, 1), (1, 1, 1), 4),
+                                          ((6, 16, 24), (1, 8, 8), 2)])
+def test_mask_at_any_allowed_alignment_with_guard_bytes(B, grid, tile, nh):
+    """The mask is written in aligned 32-byte pieces; a base that is only 16-byte aligned (the
+    contract's minimum), and rows shorter than a piece, must give the same bytes and touch nothing
+    outside the array.  A base that is not 16-byte aligned is rejected."""
+    import ctypes
+    params = [(1 + h % 2, (h % 3) - 1, [INF, 2, 3][h % 3], 1 + (h % 3), h % 2, [INF, 3][h % 2]) for h in range(nh)]
+    om, orp, oc = O.block_index_lists(params, *grid, tuple(tile))
+    nb, nnz = B.psa_mask_sizes(params, grid, tile)
+    prob = B.make_problem(nh, tile, 1.0, 0, 128)
+    n = nh * nb * nb
+    for off in (0, 16, 48, 80):
+        buf = torch.full((n + 256,), 0xEE, dtype=torch.uint8, device="cuda")
+        rp = torch.zeros(nh * nb + 1, dtype=torch.int32, device="cuda")
+        col = torch.zeros(max(nnz, 1), dtype=torch.int32, device="cuda")
+        rc = B.lib().psa_mask_build(B._params_array(params), ctypes.byref(prob), *grid, buf.data_ptr() + 64 + off,
+                                    rp.data_ptr(), col.data_ptr(), col.numel(), None)
+        assert rc == B.PSA_OK
+        torch.cuda.synchronize()
+        got = buf.cpu().numpy()
+        assert np.array_equal(got[64 + off:64 + off + n].reshape(om.shape), om), off
+        assert (got[:64 + off] == 0xEE).all() and (got[64 + off + n:] == 0xEE).all(), off
+        assert np.array_equal(rp.cpu().numpy(), orp) and np.array_equal(col.cpu().numpy()[:nnz], oc)
+    assert B.lib().psa_mask_build(B._params_array(params), ctypes.byref(prob), *grid, buf.data_ptr() + 7,
+                                  rp.data_ptr(), col.data_ptr(), col.numel(), None) == B.PSA_ERR_INVALID_ARG
