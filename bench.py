@@ -337,8 +337,8 @@ def run_ours(args, w):
                                    "frac_of_hbm_peak": mb_bytes / (mb_graph_us * 1e-6) / 1e9 / peaks["hbm_gbs"],
                                    "note": "us_per_call: back-to-back C-ABI calls incl. the host's launch cost; "
                                            "us_per_launch_in_graph: 20 captured launches replayed (GB/s uses this); one kernel "
-                                           "per call; the outputs stay in L2, the kernel is bound by launch latency and by its "
-                                           "per-row dependent instruction chains, not by HBM"}
+                                           "per call; the outputs stay in L2, the kernel is bound by launch latency and "
+                                           "instruction issue, not by HBM"}
             # ---- the same kernel with an all-covering mask (in-house dense baseline)
             Tp, Hp, Wp = -(-T // tile[0]), -(-H // tile[1]), -(-W // tile[2])
             dense_params = [(Tp, 0, 0, Hp * Wp, 0, 0)] * nh

@@ -153,12 +153,21 @@ struct HeadSets {
   int base[kMaxHeads];  // number of attended block pairs of all earlier heads
 };
 
+// Constants of the closed-form 32-bit mask window (see the kernel).  groups = temporal groups a
+// window can touch; mul / keep spread `groups` consecutive temporal bits to a spacing of S' bits
+// (bit i lands on i * S'; all partial products fall on distinct bits while groups <= S' - 1).
+struct WindowConsts {
+  unsigned long long mul, keep;
+  int groups, enabled;
+};
+
 // n / d for n < 2^16, d <= 2^11 with m = ceil(2^40 / d): exact (n * (m * d - 2^40) < 2^40)
 __device__ __forceinline__ int div_magic(int n, unsigned long long m) { return (int)(((unsigned long long)(unsigned)n * m) >> 40); }
 
-__global__ void __launch_bounds__(256)
+// (Six resident blocks per SM -- 40 registers -- let the 840 blocks of the Wan 14B shape start in one wave.)
+__global__ void __launch_bounds__(256, 6)
 mask_build_small_kernel(const HeadSets hs, const Geom g, int n_heads_here, unsigned long long magic_nb,
-                        unsigned long long magic_sp, uint8_t* __restrict__ block_mask, int* __restrict__ row_ptr,
+                        unsigned long long magic_sp, const WindowConsts wc, uint8_t* __restrict__ block_mask, int* __restrict__ row_ptr,
                         int* __restrict__ col_idx, int total_nnz) {
   const int h = blockIdx.y, tq = blockIdx.x;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
@@ -257,10 +266,33 @@ mask_build_small_kernel(const HeadSets hs, const Geom g, int n_heads_here, unsig
       return bits;
     };
     const int nchunks = len > lead ? (len - lead + 31) >> 5 : 0;
+    // Closed form of a window that stays inside the block's rows: the temporal bits tk, tk + 1, ...
+    // are spread to a spacing of S' bits by one multiplication, widened to runs of S' ones
+    // ((x << S') - x), and combined with the spatial pattern repeated with period S'; the window
+    // starts sk bits in.  A window that leaves the block's rows takes the general loop above.
+    auto periodic = [&](unsigned m) -> unsigned long long {
+      unsigned long long r = m;
+      for (int wd = Sp; wd < 64; wd <<= 1) r |= r << wd;
+      return r;
+    };
+    auto runs = [&](int tk) -> unsigned long long {
+      const unsigned long long tw = (mT >> tk) & ((1ull << wc.groups) - 1ull);
+      const unsigned long long spread = (tw * wc.mul) & wc.keep;
+      return (spread << Sp) - spread;
+    };
+    const unsigned long long runs0 = runs(0);
     for (int c = threadIdx.x; c < nchunks; c += blockDim.x) {
       const int r = lead + 32 * c;
-      int n;
-      const unsigned bits = gen(r, 32, &n);
+      int n = 32;
+      unsigned bits;
+      const int sq = div_magic(r, magic_nb), kb = r - sq * NB;
+      if (wc.enabled && (kb + 32 <= NB || sq + 1 < Sp)) {
+        const int tk = div_magic(kb, magic_sp), sk = kb - tk * Sp;
+        bits = (unsigned)((runs(tk) & periodic(rowS(sq))) >> sk);
+        if (kb + 32 > NB) bits |= (unsigned)(runs0 & periodic(rowS(sq + 1))) << (NB - kb);   // on into the next row
+      } else {
+        bits = gen(r, 32, &n);
+      }
       if (n == 32) {
         uint32_t w[8];
 #pragma unroll
@@ -331,9 +363,20 @@ cudaError_t launch_mask_build(const HeadParamsArray& hp, const int* head_bases, 
     const unsigned long long two40 = 1ull << 40;
     const unsigned long long magic_nb = (two40 + (unsigned long long)g.NB - 1ull) / (unsigned long long)g.NB;
     const unsigned long long magic_sp = (two40 + (unsigned long long)g.Sp - 1ull) / (unsigned long long)g.Sp;
+    // the closed-form window needs its partial products on distinct bits and at most one row end per window
+    WindowConsts wc;
+    wc.groups = (g.Sp - 1 + 31) / g.Sp + 1;
+    wc.enabled = (wc.groups <= g.Sp - 1 && g.NB >= 32) ? 1 : 0;
+    wc.mul = 0;
+    wc.keep = 0;
+    if (wc.enabled)
+      for (int i = 0; i < wc.groups; ++i) {
+        wc.mul |= 1ull << (i * (g.Sp - 1));
+        if (i * g.Sp < 64) wc.keep |= 1ull << (i * g.Sp);
+      }
     dim3 grid(g.Tp, n_heads_here);   // one block per (head, temporal query coordinate)
     mask_build_small_kernel<<<grid, 256, 0, stream>>>(
-        hs, g, n_heads_here, magic_nb, magic_sp, block_mask, row_ptr, col_idx, total_nnz_through_chunk);
+        hs, g, n_heads_here, magic_nb, magic_sp, wc, block_mask, row_ptr, col_idx, total_nnz_through_chunk);
     ++*launches;
     return cudaGetLastError();
   }
