@@ -100,3 +100,15 @@ def test_mask_at_any_allowed_alignment_with_guard_bytes(B, grid, tile, nh):
         assert np.array_equal(rp.cpu().numpy(), orp) and np.array_equal(col.cpu().numpy()[:nnz], oc)
     assert B.lib().psa_mask_build(B._params_array(params), ctypes.byref(prob), *grid, buf.data_ptr() + 7,
                                   rp.data_ptr(), col.data_ptr(), col.numel(), None) == B.PSA_ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("grid", [(64, 4, 8), (5, 1, 7), (6, 2, 3), (9, 2, 4), (40, 1, 1), (33, 3, 5), (2, 4, 8)])
+def test_extreme_block_grids_of_the_register_path(B, grid):
+    """Token-granular masks that sit on the limits of the small-grid kernel: 64 temporal x 32 spatial
+    coordinates, spatial extents around the threshold of its closed-form mask window (7 and 8 use it,
+    6 and 1 do not), rows shorter than one 32-byte piece."""
+    T, H, W = grid
+    params = [(1 + h % 3, (h % 5) - 2, [INF, 2, 3, 5][h % 4], 1 + (h % 2), (h % 3) - 1, [INF, 3, 5, 6][(h // 2) % 4])
+              for h in range(6)]
+    params += [(T, 0, INF, H * W, 0, INF), (1, 0, INF, 1, 0, INF), (2, T, INF, 1, 0, INF)]   # all-pass, diagonal, empty
+    _check(B, params, grid, (1, 1, 1))
