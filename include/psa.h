@@ -140,7 +140,8 @@ int psa_attn_fwd_noalloc(const void* q, const void* k, const void* v, void* out,
  * outermost dimension of the layout the call is pipelined over chunks of heads (20 by default,
  * from a measured sweep; the environment variable PSA_HOST_CHUNKS overrides it) on two internal
  * helper streams: the next chunk is copied in and the previous one copied out while a chunk
- * computes.
+ * computes.  Chunks are contiguous head ranges but need not run in head order: the call opens
+ * with single heads and keeps the two heads with the fewest attended block pairs for the end.
  * Each staging buffer must hold the full strided extent of its tensor:
  * (n_heads-1)*stride_head + (L-1)*stride_token + head_dim elements. */
 int psa_attn_fwd_host(const void* q, const void* k, const void* v, void* out, float* lse,

@@ -686,7 +686,7 @@ int psa_attn_fwd_host(const void* q, const void* k, const void* v, void* out, fl
   // Chunk size: the call is bound by the host-to-device copies, so what is exposed is the first
   // chunk's copy-in and the last chunk's compute and copy-out -- both shrink with the chunk.
   int want = host_chunks();
-  if (want > kHostChunks) want = kHostChunks;
+  if (want > kHostChunks - 8) want = kHostChunks - 8;   // single-head edge chunks and broken runs add a few
   const int n_chunks = prob->n_heads < want ? prob->n_heads : want;
   const int per = (prob->n_heads + n_chunks - 1) / n_chunks;
   // everything enqueued on `stream` before this call precedes the first copy
@@ -694,14 +694,44 @@ int psa_attn_fwd_host(const void* q, const void* k, const void* v, void* out, fl
   if (cudaStreamWaitEvent(pipe->h2d, pipe->ev_start, 0) != cudaSuccess) return PSA_ERR_CUDA;
   if (cudaStreamWaitEvent(pipe->d2h, pipe->ev_start, 0) != cudaSuccess) return PSA_ERR_CUDA;
   // The first and the last chunks are the exposed ones, so the call starts and ends with
-  // single-head chunks (two at each end, when the regular chunk is larger than that).
+  // single-head chunks (two at each end, when the regular chunk is larger than that), and the two
+  // heads with the fewest attended block pairs (the shortest kernels) are kept for the end: what
+  // remains after the last byte has arrived is the lightest head's kernel and its copy-out.
   const int n_edge = (per >= 2 && prob->n_heads >= 4 * per) ? 2 : 0;
-  int c = 0;
-  for (int h0 = 0, nh = 0; h0 < prob->n_heads; h0 += nh, ++c) {
-    const int left = prob->n_heads - h0;
-    if (h0 < n_edge || left <= n_edge) nh = 1;
-    else nh = left - n_edge < per ? left - n_edge : per;
-    if (c >= kHostChunks) return PSA_ERR_UNSUPPORTED;
+  struct Chunk { int h0, nh; };
+  Chunk chunks[kHostChunks];
+  int n_list = 0;
+  int last1 = -1, last2 = -1;   // lightest and second-lightest head
+  if (n_edge) {
+    Geom g;
+    const int rcg = make_geom(prob, T, H, W, true, &g);
+    if (rcg != PSA_OK) return rcg;
+    long long w1 = 0, w2 = 0;
+    for (int h = 0; h < prob->n_heads; ++h) {
+      if (!valid_params(head_params[h])) return PSA_ERR_INVALID_ARG;
+      const long long w = head_nnz(head_params[h], g);
+      if (last1 < 0 || w < w1) { last2 = last1; w2 = w1; last1 = h; w1 = w; }
+      else if (last2 < 0 || w < w2) { last2 = h; w2 = w; }
+    }
+  }
+  {
+    int singles = n_edge;   // single-head chunks still to open the call with
+    int h = 0;
+    while (h < prob->n_heads) {
+      if (h == last1 || h == last2) { ++h; continue; }
+      int nh = 1;
+      if (singles > 0) --singles;
+      else
+        while (nh < per && h + nh < prob->n_heads && h + nh != last1 && h + nh != last2) ++nh;
+      if (n_list >= kHostChunks - 2) return PSA_ERR_UNSUPPORTED;
+      chunks[n_list++] = Chunk{h, nh};
+      h += nh;
+    }
+    if (last2 >= 0) chunks[n_list++] = Chunk{last2, 1};
+    if (last1 >= 0) chunks[n_list++] = Chunk{last1, 1};
+  }
+  for (int c = 0; c < n_list; ++c) {
+    const int h0 = chunks[c].h0, nh = chunks[c].nh;
     const size_t off = (size_t)h0 * prob->stride_head;                       // elements
     const size_t bytes = ((size_t)(nh - 1) * prob->stride_head + head_span) * 2;
     const uint16_t *hq = static_cast<const uint16_t*>(q) + off, *hk = static_cast<const uint16_t*>(k) + off,

@@ -205,6 +205,30 @@ def test_host_tensor_entry_point_matches_device_call(B, pinned):
         assert torch.equal(hlse.view(torch.int32), ref_lse.cpu().view(torch.int32))
 
 
+def test_host_tensor_call_with_reordered_chunks(B):
+    """40 heads of very different weight: the host call pipelines 2-head chunks, opens with single
+    heads and keeps the two lightest heads for the end (here heads 17 and 5, in the middle of runs);
+    the result must be the device call's, bit for bit."""
+    grid, tile, nh = (4, 16, 16), (1, 16, 16), 40
+    L = 4 * 16 * 16
+    params = [(1 + (h % 4), (h % 3) - 1, INF, 1, 0, INF) for h in range(nh)]
+    params[17] = (1, 3, INF, 1, 0, INF)     # one attended block pair per row at most: the lightest
+    params[5] = (1, 2, INF, 1, 0, INF)      # the second lightest
+    bits = {n: WL.tensor_bits(0x7D, n, nh, L, threads=1) for n in ("q", "k", "v")}
+    host = {n: torch.from_numpy(bits[n].view(np.int16)).view(torch.bfloat16) for n in bits}
+    dev = {n: host[n].cuda() for n in host}
+    ref_out, ref_lse = B.psa_attn_fwd(dev["q"], dev["k"], dev["v"], params, grid, tile, SCALE)
+    assert B.psa_last_device_status()[0] == 0
+    hq, hk, hv = (host[n].pin_memory() for n in ("q", "k", "v"))
+    hout = torch.full_like(hq, float("nan")).pin_memory()
+    hlse = torch.full((nh, L), float("nan"), dtype=torch.float32).pin_memory()
+    staging = tuple(torch.empty_like(dev["q"]) for _ in range(4)) + (torch.empty((nh, L), dtype=torch.float32, device="cuda"),)
+    B.psa_attn_fwd_host(hq, hk, hv, hout, hlse, staging, params, grid, tile, SCALE)
+    assert B.psa_last_device_status()[0] == 0
+    assert torch.equal(hout.view(torch.int16), ref_out.cpu().view(torch.int16))
+    assert torch.equal(hlse.view(torch.int32), ref_lse.cpu().view(torch.int32))
+
+
 def test_more_heads_than_one_launch_carries(B):
     """130 heads: the library splits the call into launches of at most 128 heads."""
     grid, tile, nh = (2, 16, 16), (1, 16, 16), 130
